@@ -1,0 +1,351 @@
+"""Pins for the CPU oracle: closed forms, invariants, hand-worked values, library
+routines on special cases and brute force on tiny inputs.  None of these retype
+the oracle's own butterfly / quantizer code: each checks it against something
+the mathematics fixes independently."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import hbl_oracle as orc
+from paper_2504_18415_b200 import workloads as wl
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_cases.json")))
+EPS = 1e-5
+PRECS = (32, 64)
+
+
+def Phi(z):
+    return 0.5 * (1.0 + math.erf(z / math.sqrt(2.0)))
+
+
+# ------------------------------------------------------------------ Hadamard
+def popcount_matrix(n):
+    """Entry closed form of the Sylvester matrix: H[i,j] = (-1)^popcount(i&j)."""
+    H = np.empty((n, n))
+    for i in range(n):
+        for j in range(n):
+            H[i, j] = -1.0 if bin(i & j).count("1") & 1 else 1.0
+    return H
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 16, 32, 64])
+def test_hadamard_matches_popcount_closed_form(n):
+    rng = np.random.default_rng(n)
+    x = rng.standard_normal((5, n)).astype(np.float32)
+    want = x.astype(np.float64) @ popcount_matrix(n).T / math.sqrt(n)
+    got = orc.hadamard(x)
+    assert np.allclose(got, want, rtol=0, atol=1e-13 * n)
+
+
+@pytest.mark.parametrize("n", [2, 16, 256])
+def test_hadamard_matches_kronecker_and_scipy(n):
+    from scipy.linalg import hadamard as scipy_hadamard
+    H2 = np.array([[1.0, 1.0], [1.0, -1.0]])
+    H = np.array([[1.0]])
+    while H.shape[0] < n:
+        H = np.kron(H2, H)          # the recursion of Eq. 4 without the 1/sqrt(2)
+    assert np.array_equal(H, scipy_hadamard(n).astype(np.float64))
+    got = orc.hadamard(np.eye(n, dtype=np.float32)) * math.sqrt(n)   # rows = H e_i
+    assert np.allclose(got, H, atol=1e-12)
+    assert np.allclose(got @ got.T, n * np.eye(n), atol=1e-9)        # H H^T = n I
+
+
+@pytest.mark.parametrize("case", GOLD["hadamard"], ids=lambda c: c["cite"])
+def test_hadamard_hand_values(case):
+    x = np.array([case["x"]], dtype=np.float32)
+    got = orc.hadamard(x)[0] * math.sqrt(len(case["x"]))
+    assert np.allclose(got, case["xr_times_sqrt_n"], atol=1e-12)
+
+
+@pytest.mark.parametrize("n", [8, 512, 4096, 16384])
+def test_hadamard_invariants(n):
+    rng = np.random.default_rng(n + 1)
+    x = rng.standard_normal((3, n)).astype(np.float32)
+    y = orc.hadamard(x)
+    # Parseval (orthonormal)
+    assert np.allclose((y ** 2).sum(1), (x.astype(np.float64) ** 2).sum(1), rtol=1e-12)
+    # involution: the transform applied twice returns the input (inputs kept fp32-exact)
+    y32 = y.astype(np.float32)
+    back = orc.hadamard(y32)
+    assert np.allclose(back, x, atol=1e-5 * np.abs(x).max())
+    # e_0 -> 1/sqrt(n); all-ones -> sqrt(n) e_0
+    e0 = np.zeros((1, n), np.float32); e0[0, 0] = 1
+    assert np.allclose(orc.hadamard(e0), 1 / math.sqrt(n), atol=1e-15)
+    ones = orc.hadamard(np.ones((1, n), np.float32))[0]
+    assert abs(ones[0] - math.sqrt(n)) < 1e-10 and np.abs(ones[1:]).max() < 1e-10
+    # e_j -> column j of H: sign pattern (-1)^popcount(i&j), natural order
+    j = n // 2 + 1 if n > 2 else 1
+    ej = np.zeros((1, n), np.float32); ej[0, j] = 1
+    col = orc.hadamard(ej)[0] * math.sqrt(n)
+    idx = np.arange(n)
+    pc = np.array([bin(int(i) & j).count("1") & 1 for i in idx])
+    assert np.array_equal(col, np.where(pc == 1, -1.0, 1.0))
+    # linearity (exact inputs)
+    a = np.float32(0.5); b = np.float32(-2.0)
+    lin = orc.hadamard((a * x[0:1] + b * x[1:2]).astype(np.float32))
+    # (a*x0+b*x1 is rounded to fp32 before the call; compare against the rounded input's transform)
+    assert np.allclose(lin, a * y[0:1] + b * y[1:2], atol=1e-5)
+
+
+def test_hadamard_rejects_non_power_of_two():
+    with pytest.raises(RuntimeError):
+        orc.hadamard(np.zeros((1, 12), np.float32))
+
+
+# ------------------------------------------------------------------ quantizers
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("case", GOLD["int4"], ids=lambda c: c["cite"])
+def test_int4_hand_values(case, prec):
+    x = np.array([case["x"]], dtype=np.float64)
+    q, v, s, st = orc.act_quant(x, 4, EPS, prec)
+    assert q[0].tolist() == case["codes"]
+    assert abs(st[0] - case["beta"]) < 1e-6
+    assert abs(s[0] - case["s"]) < 1e-6
+    assert np.all(np.isfinite(v))
+
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("case", GOLD["int8"], ids=lambda c: c["cite"])
+def test_int8_hand_values(case, prec):
+    x = np.array([case["x"]], dtype=np.float64)
+    q, v, s, st = orc.act_quant(x, 8, case.get("eps", EPS), prec)
+    assert q[0].tolist() == case["codes"]
+    assert abs(st[0] - case["gamma"]) < 1e-6
+    assert abs(s[0] - case["s"]) < 1e-6
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_int4_code_distribution_on_gaussian(prec):
+    """For x ~ N(0,1), beta -> sqrt(2/pi); the code histogram follows from Phi."""
+    K, T = 16384, 64
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((T, K))
+    q, v, s, st = orc.act_quant(x, 4, EPS, prec)
+    beta = math.sqrt(2 / math.pi)
+    assert abs(st.mean() - beta) < 2e-3
+    c = math.sqrt(7) / beta                      # v = c * x
+    def p_code(k):
+        lo = -math.inf if k == -8 else (k - 0.5) / c
+        hi = math.inf if k == 7 else (k + 0.5) / c
+        return Phi(hi) - Phi(lo)
+    n = q.size
+    for k in range(-8, 8):
+        want = p_code(k)
+        got = np.count_nonzero(q == k) / n
+        assert abs(got - want) < 5 * math.sqrt(want * (1 - want) / n) + 2e-4, (k, got, want)
+    assert abs(p_code(7) - 0.0250) < 2e-4 and abs(p_code(-8) - 0.0119) < 2e-4
+    assert q.min() == -8 and q.max() == 7
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_int8_never_reaches_minus_128_and_hits_127(prec):
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((32, 1024)) * 3.0
+    q, v, s, st = orc.act_quant(x, 8, EPS, prec)
+    assert q.min() >= -127 and q.max() <= 127
+    # the absmax entry of every token maps to +-127
+    am = np.abs(x).argmax(1)
+    assert np.all(np.abs(q[np.arange(32), am].astype(int)) == 127)
+    assert np.allclose(st, np.abs(x).max(1), rtol=1e-6)
+    assert np.allclose(s, st / 127.0, rtol=1e-12)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_quantizer_dequant_error_bound(bits):
+    """Away from clipping, |s*q - x*stat/(stat+eps)| <= s/2 (round to nearest)."""
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((8, 2048))
+    q, v, s, st = orc.act_quant(x, bits, EPS, 64)
+    hi = 127 if bits == 8 else 7
+    lo = -128 if bits == 8 else -8
+    inside = (v > lo - 0.5) & (v < hi + 0.5)
+    err = np.abs(s[:, None] * q - x * (st / (st + EPS))[:, None])
+    assert np.all(err[inside] <= 0.5 * np.broadcast_to(s[:, None], err.shape)[inside] * (1 + 1e-9))
+    assert np.all(q[v >= hi + 0.5] == hi) and np.all(q[v <= lo - 0.5] == lo)
+
+
+def test_bits_must_be_4_or_8():
+    with pytest.raises(RuntimeError):
+        orc.act_quant(np.zeros((1, 4)), 5, EPS, 64)
+
+
+# ------------------------------------------------------------------ ternary weights
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("case", GOLD["ternary"], ids=lambda c: c["cite"])
+def test_ternary_hand_values(case, prec):
+    wt, alpha = orc.weight_quant(np.array(case["W"], np.float32), EPS, prec)
+    assert abs(float(alpha) - case["alpha"]) < 1e-7
+    assert wt.tolist() == case["wt"]
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_ternary_statistics_on_gaussian_latents(prec):
+    sigma = 0.02
+    W = wl.rows("latent", 123, 1, 2048, 0, 1024)
+    wt, alpha = orc.weight_quant(W, EPS, prec)
+    assert abs(float(alpha) / sigma - math.sqrt(2 / math.pi)) < 2e-3
+    # w = 0 iff |W| < (alpha+eps)/2  (up to the tie)
+    z = 0.5 * (float(alpha) + EPS) / sigma
+    p0 = 2 * Phi(z) - 1
+    n = wt.size
+    assert abs(np.count_nonzero(wt == 0) / n - p0) < 5 * math.sqrt(p0 * (1 - p0) / n)
+    assert abs(p0 - 0.310) < 2e-3
+    assert abs(np.count_nonzero(wt == 1) / n - (1 - p0) / 2) < 3e-3
+    assert set(np.unique(wt).tolist()) == {-1, 0, 1}
+    # independent restatement of the decision on a sample, in exact rational-free form:
+    # |W| > (alpha+eps)/2 <=> |w| = 1 and sign(w) = sign(W)
+    thr = 0.5 * (np.float64(alpha) + EPS)
+    far = np.abs(np.abs(W.astype(np.float64)) - thr) > 1e-7
+    assert np.array_equal(wt[far], (np.sign(W) * (np.abs(W.astype(np.float64)) > thr))[far].astype(np.int8))
+
+
+def test_ternary_alpha_is_fp64_mean_rounded_once():
+    W = wl.rows("latent", 5, 9, 512, 0, 512)
+    _, alpha = orc.weight_quant(W, EPS, 64)
+    want = np.float32(math.fsum(np.abs(W.astype(np.float64)).ravel().tolist()) / W.size)
+    assert alpha == want
+
+
+# ------------------------------------------------------------------ contraction and rescale
+def test_gemm_matches_fp64_matmul_and_special_cases():
+    rng = np.random.default_rng(11)
+    q = rng.integers(-128, 128, size=(7, 96), dtype=np.int8)
+    wt = rng.integers(-1, 2, size=(13, 96), dtype=np.int8)
+    acc = orc.gemm(q, wt)
+    assert np.array_equal(acc, (q.astype(np.float64) @ wt.astype(np.float64).T).astype(np.int64))
+    assert np.array_equal(orc.gemm(q, np.ones((3, 96), np.int8)), np.repeat(q.astype(np.int64).sum(1)[:, None], 3, 1))
+    onehot = np.zeros((96, 96), np.int8); onehot[np.arange(96), np.arange(96)[::-1]] = -1
+    assert np.array_equal(orc.gemm(q, onehot), -q[:, ::-1].astype(np.int32))
+    # extreme magnitudes: K=16384 of (-128)*(-1) stays inside int32
+    K = 16384
+    assert orc.gemm(np.full((1, K), -128, np.int8), np.full((1, K), -1, np.int8))[0, 0] == 128 * K
+
+
+def test_rescale_rounds_once_to_bf16():
+    import torch
+    acc = np.array([[1, 3, -5, 257, 129, 131, 0, 7]], dtype=np.int32)
+    yb, y64 = orc.rescale(acc, np.array([1.0]), 1.0)
+    # 257 = 1.00000001b*2^8 lies exactly between 256 and 258 -> even significand (256);
+    # 129 (between 128 and 130 in bf16? no: 129 = 10000001b is exact, 8 bits) stays.
+    want = torch.tensor(acc[0].astype(np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(yb[0], want)
+    assert orc.bf16_bits_to_f32(yb)[0].tolist() == [1.0, 3.0, -5.0, 256.0, 129.0, 131.0, 0.0, 7.0]
+    # ties at the 9th significand bit go to even: 1+2^-8 -> 1, 1+3*2^-8 -> 1+2^-6
+    yb, _ = orc.rescale(np.array([[1 << 20]], np.int32), np.array([(1 + 2.0 ** -8) / (1 << 20)]), 1.0)
+    assert orc.bf16_bits_to_f32(yb)[0, 0] == 1.0
+    yb, _ = orc.rescale(np.array([[1 << 20]], np.int32), np.array([(1 + 3 * 2.0 ** -8) / (1 << 20)]), 1.0)
+    assert orc.bf16_bits_to_f32(yb)[0, 0] == 1.0 + 2.0 ** -6
+    # a value just above a tie must round up even though (float) would land on the tie first
+    v = 1 + 2.0 ** -8 + 2.0 ** -40
+    yb, _ = orc.rescale(np.array([[1]], np.int32), np.array([v]), 1.0)
+    assert orc.bf16_bits_to_f32(yb)[0, 0] == 1.0 + 2.0 ** -7
+    # random values against torch's fp32->bf16 on fp32-exact products
+    rng = np.random.default_rng(3)
+    acc = rng.integers(-100000, 100000, size=(4, 64)).astype(np.int32)
+    yb, y64 = orc.rescale(acc, np.array([0.5, 0.25, 2.0, 1.0]), 0.125)
+    want = torch.tensor(y64.astype(np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(yb, want)
+
+
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("case", GOLD["layer"], ids=lambda c: c["cite"])
+def test_layer_hand_values(case, prec):
+    W = np.array(GOLD["ternary"][0]["W"], np.float32)
+    wt, alpha = orc.weight_quant(W, EPS, prec)
+    x = np.array([case["x"]], np.float32)
+    out = orc.forward(x, wt, alpha, case["bits"], bool(case["use_hadamard"]), EPS, prec, want_stages=True)
+    assert out["codes"][0].tolist() == case["codes"]
+    assert out["acc"][0].tolist() == case["acc"]
+    assert np.allclose(out["y64"][0], case["y"], atol=2e-5)
+    import torch
+    want_bf16 = torch.tensor(case["y"], dtype=torch.float64).to(torch.float32).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(orc.bf16_bits_to_f32(out["y_bits"])[0], want_bf16)
+
+
+def test_forward_equals_its_stages_and_dense_definition():
+    """Eq. 7 written densely: y = (alpha*W_t) @ (s*q), with x_r from the dense popcount matrix."""
+    n, N, T = 64, 24, 5
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((T, n)).astype(np.float32)
+    x[:, 3] *= 40
+    W = (rng.standard_normal((N, n)) * 0.02).astype(np.float32)
+    wt, alpha = orc.weight_quant(W, EPS, 64)
+    out = orc.forward(x, wt, alpha, 4, True, EPS, 64, want_stages=True)
+    xr = x.astype(np.float64) @ popcount_matrix(n) / math.sqrt(n)
+    beta = np.abs(xr).mean(1, keepdims=True)
+    q = np.clip(np.rint(xr * math.sqrt(7) / (beta + EPS)), -8, 7)
+    y = (q * beta / math.sqrt(7)) @ (float(alpha) * wt.astype(np.float64)).T
+    assert np.array_equal(out["codes"], q.astype(np.int8))
+    assert np.allclose(out["y64"], y, rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------------ properties of the layer
+def test_rotation_identity_without_quantization():
+    """W x = (W H)(H x): the transform is orthogonal, so rotating both sides changes nothing."""
+    n = 256
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((4, n)).astype(np.float32)
+    W = rng.standard_normal((16, n)).astype(np.float32)
+    lhs = x.astype(np.float64) @ W.astype(np.float64).T
+    rhs = orc.hadamard(x) @ orc.hadamard(W).T
+    assert np.allclose(lhs, rhs, atol=1e-9)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_token_scaling_and_permutation(bits):
+    wlc = wl.CONFIG1
+    x = wlc.x(0, 8)
+    wt, alpha = orc.weight_quant(wlc.w_latent(), EPS, 64)
+    base = orc.forward(x, wt, alpha, bits, True, EPS, 64, want_stages=True)
+    sc = orc.forward((x * np.float32(4.0)), wt, alpha, bits, True, EPS, 64, want_stages=True)
+    assert np.array_equal(base["codes"], sc["codes"])          # eps shift is far below any boundary here
+    assert np.allclose(sc["y64"], 4.0 * base["y64"], rtol=1e-12)
+    perm = np.array([3, 1, 7, 0, 2, 6, 5, 4])
+    pm = orc.forward(x[perm], wt, alpha, bits, True, EPS, 64)
+    assert np.array_equal(pm["y_bits"], base["y_bits"][perm])
+
+
+def test_hadamard_removes_outlier_channels_on_the_workloads():
+    """Section 2.1's qualitative claim on the synthetic stand-ins: after the transform the
+    per-token max/mean ratio collapses and INT4 round-trip error drops."""
+    for cfg in (wl.CONFIG1, wl.CONFIG2, wl.CONFIG3):
+        x = cfg.x(0, 16)
+        xr = orc.hadamard(x)
+        r_before = (np.abs(x).max(1) / np.abs(x).mean(1)).mean()
+        r_after = (np.abs(xr).max(1) / np.abs(xr).mean(1)).mean()
+        assert r_after < 0.25 * r_before, (cfg.name, r_before, r_after)
+        assert r_after < 8.0                      # Gaussian-like: max/mean ~ 4-6 for these K
+        def rel_mse(v):
+            q, _, s, _ = orc.act_quant(v, 4, EPS, 64)
+            return (((q * s[:, None]) - v) ** 2).sum() / (v ** 2).sum()
+        assert rel_mse(xr) < 0.5 * rel_mse(x.astype(np.float64)), cfg.name
+
+
+def test_layer_tracks_the_unquantized_product_with_int8():
+    cfg = wl.CONFIG1
+    x = cfg.x(0, 16)
+    wt, alpha = orc.weight_quant(cfg.w_latent(), EPS, 64)
+    out = orc.forward(x, wt, alpha, 8, True, EPS, 64)
+    ref = orc.hadamard(x) @ (float(alpha) * wt.astype(np.float64)).T
+    rel = np.linalg.norm(out["y64"] - ref) / np.linalg.norm(ref)
+    assert rel < 0.02
+
+
+# ------------------------------------------------------------------ generators
+def test_workload_rows_are_reproducible_and_blockwise():
+    a = wl.rows("attn_out", 2, 1, 2048, 0, 200, "bf16")
+    b = wl.rows("attn_out", 2, 1, 2048, 130, 50, "bf16")
+    assert np.array_equal(a[130:180], b)
+    assert np.array_equal(wl.round_to_bf16(a)[0], a)
+    ch = wl.outlier_channels(2, 1, 2048, 0.005)
+    assert len(ch) == 10
+    col_rms = np.sqrt((a ** 2).mean(0))
+    assert col_rms[ch].min() > 10 * np.median(col_rms)
+    assert wl.CONFIG1.x(0, 64).shape == (64, 512)
+    assert len(wl.outlier_channels(0, 1, 512, 0.01)) == 5
+    assert len(wl.outlier_channels(3, 1, 8192, 0.002)) == 16
+    w = wl.CONFIG2.w_latent(0, 64)
+    assert abs(w.std() - 0.02) < 5e-4
