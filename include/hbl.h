@@ -1,0 +1,146 @@
+/* hbl.h -- C ABI of the H-BitLinear forward pass for NVIDIA B200 (sm_100a).
+ *
+ * The layer (BitNet v2, section 2.1, Eq. 1-7), for T tokens x[T,K] and latent
+ * weights W[N,K] (row-major, K = in_dim, N = out_dim):
+ *
+ *   alpha = mean|W|,  W_t = RoundClip(W/(alpha+eps), -1, 1)             (Eq. 1-2)
+ *   x_r   = H_m x   (orthonormal Sylvester-Hadamard, K = 2^m)            (Eq. 3-4)
+ *   INT8: gamma = max|x_r|,  q = RoundClip(127/(gamma+eps) x_r, -128, 127), s = gamma/127   (Eq. 5)
+ *   INT4: beta  = mean|x_r|, q = RoundClip(sqrt(7)/(beta+eps) x_r, -8, 7),   s = beta/sqrt(7) (Eq. 6)
+ *   y[t,o] = alpha * s_t * sum_k W_t[o,k] q[t,k]   -> bf16                (Eq. 7)
+ *
+ * round() is round-half-to-even.  eps is an explicit argument (> 0).
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller, unless a
+ *     parameter is documented as a host pointer.  The library allocates no
+ *     device memory and frees none; scratch space is the caller's `workspace`.
+ *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*;
+ *     NULL is the default stream).  No entry point synchronises except
+ *     hbl_check_status.
+ *   - Every call returns an hbl_status_t.  Argument errors are found on the
+ *     host before anything is launched.  A device-side wait that runs out
+ *     records HBL_ERR_TIMEOUT in a status word that hbl_check_status reads.
+ *   - Alignment: all buffers 16 bytes; workspace 1024 bytes.
+ *   - Shapes: in_dim % 128 == 0, out_dim % 16 == 0, in_dim <= 32768,
+ *     tokens >= 0 (0 is a no-op that returns HBL_OK).
+ */
+#ifndef HBL_H_
+#define HBL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  HBL_OK = 0,
+  HBL_ERR_NULL = 1,        /* a required pointer is NULL */
+  HBL_ERR_SHAPE = 2,       /* a dimension is negative, zero where not allowed, or not a supported multiple */
+  HBL_ERR_NOT_POW2 = 3,    /* use_hadamard with in_dim not a power of two (Eq. 4 needs n = 2^m) */
+  HBL_ERR_BITS = 4,        /* bits not 4 or 8 */
+  HBL_ERR_ALIGN = 5,       /* a pointer is not aligned as required */
+  HBL_ERR_WORKSPACE = 6,   /* workspace smaller than hbl_workspace_bytes() says */
+  HBL_ERR_EPS = 7,         /* eps <= 0 or not finite */
+  HBL_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed (launch error, no device) */
+  HBL_ERR_TIMEOUT = 9,     /* a bounded device-side wait expired */
+  HBL_ERR_FORMAT = 10,     /* unknown dtype / path id */
+  HBL_ERR_TOO_LARGE = 11   /* size beyond a stated maximum */
+} hbl_status_t;
+
+typedef enum { HBL_F32 = 0, HBL_BF16 = 1 } hbl_dtype_t;
+
+/* Which contraction kernel hbl_forward / hbl_gemm_i32 use. */
+typedef enum {
+  HBL_PATH_AUTO = 0,       /* by token count */
+  HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers); tokens <= 64 */
+  HBL_PATH_TENSOR = 2      /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
+} hbl_path_t;
+
+const char* hbl_status_string(int status);
+
+/* Bytes of the packed ternary weight tensor for W[out_dim, in_dim]: 2 bits per
+ * weight, stored as u = w + 1 in {0,1,2}.  Layout: tiles of 16 rows x 128
+ * columns, 512 bytes each, ordered [row tile][column tile]; inside a tile, 32
+ * groups of four 32-bit words; word j of group l holds the 16 weights with
+ * rows 16*tile + (l>>2) + 8*(i&1), columns 128*ctile + 32*j + 16*(i>>1) + 4*(l&3) + b
+ * (i = 0..3, b = 0..3) at bit position 8*b + 2*i.  Returns 0 on bad shapes. */
+size_t hbl_packed_weight_bytes(int out_dim, int in_dim);
+
+/* Scratch bytes hbl_forward needs for up to max_tokens tokens (any bits, any path). */
+size_t hbl_workspace_bytes(int max_tokens, int in_dim, int out_dim);
+
+/* Scratch bytes hbl_quantize_weights needs. */
+size_t hbl_quantize_weights_workspace_bytes(int out_dim, int in_dim);
+
+/* Eq. 1-2.  W_latent: [out_dim, in_dim] row-major, fp32 or bf16.  Writes the
+ * packed ternary tensor (hbl_packed_weight_bytes) and the fp32 alpha (device,
+ * one float).  alpha is the fp64-accumulated mean rounded once to fp32; the
+ * ternary decision is rint(W / (alpha + eps)) in IEEE fp32. */
+int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_dim, float eps,
+                         void* W_packed, float* alpha, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/* Eq. 3-7: the layer's forward pass for `tokens` tokens.
+ *   x         [tokens, in_dim] fp32 or bf16
+ *   W_packed  from hbl_quantize_weights;  alpha: device pointer to its scale
+ *   bits      4 (Eq. 6) or 8 (Eq. 5);  use_hadamard: 1 applies Eq. 3-4 first
+ *   y         [tokens, out_dim] bf16 (written)
+ *   path      an hbl_path_t
+ * The intermediate codes never leave the workspace. */
+int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim,
+                const void* W_packed, const float* alpha, int out_dim,
+                int bits, int use_hadamard, float eps, void* y,
+                void* workspace, size_t workspace_bytes, int path, void* stream);
+
+/* The seven projections of a LLaMA-like decoder block (section 2): q, k, v and
+ * up, gate are plain BitLinear layers (no transform) that share one quantized
+ * input each; o and down are H-BitLinear layers (Hadamard on).  Every input is
+ * supplied by the caller; attention, RoPE, SwishGLU and residuals are not part
+ * of this call.  alpha7: device array of the seven per-tensor alphas in the
+ * order q, k, v, o, up, gate, down. */
+typedef struct {
+  const void *x_attn_in, *x_o_in, *x_ffn_in, *x_down_in; /* [T,H] [T,H] [T,H] [T,F] */
+  const void *Wq, *Wk, *Wv, *Wo, *Wup, *Wgate, *Wdown;    /* packed ternary */
+  const float* alpha7;
+  void *yq, *yk, *yv, *yo, *yup, *ygate, *ydown;          /* bf16 outputs */
+  int tokens, hidden, ffn, bits, x_dtype;
+  float eps;
+} hbl_block_t;
+
+size_t hbl_block_workspace_bytes(int max_tokens, int hidden, int ffn);
+int hbl_block_forward(const hbl_block_t* block /* host pointer */, void* workspace,
+                      size_t workspace_bytes, int path, void* stream);
+
+/* Synchronises `stream`, returns the first device-side error recorded since the
+ * last call (HBL_OK if none) and clears it. */
+int hbl_check_status(void* stream);
+
+/* ---- stage-level entry points (the same kernels, exposed one step at a time) ---- */
+
+/* Eq. 3-4 alone: xr_out[T,K] fp32 = H_m x, orthonormal, natural order. */
+int hbl_hadamard_f32(const void* x, int x_dtype, int tokens, int in_dim, float* xr_out, void* stream);
+
+/* Eq. 3-6: transform (optional), per-token statistic, quantize.  codes_out: int8
+ * [T,K], one code per byte; scale_out: fp32 [T] (s_t); codesum_out: int32 [T],
+ * sum_k q[t,k] (may be NULL). */
+int hbl_quantize_act(const void* x, int x_dtype, int tokens, int in_dim, int bits, int use_hadamard,
+                     float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out, void* stream);
+
+/* Eq. 7's contraction alone: acc_out[T,N] int32 = sum_k W_t[o,k] * codes[t,k], exact.
+ * codes: int8 [T,K].  codesum: int32 [T] (sum of each token's codes; required
+ * by the streaming path, ignored by the tensor path; may be NULL with
+ * HBL_PATH_TENSOR).  workspace: hbl_workspace_bytes(T,K,N). */
+int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in_dim,
+                 const void* W_packed, int out_dim, int32_t* acc_out,
+                 void* workspace, size_t workspace_bytes, int path, void* stream);
+
+/* Packed ternary -> int8 [N,K] row-major, values in {-1,0,1}. */
+int hbl_unpack_weights(const void* W_packed, int out_dim, int in_dim, int8_t* w_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HBL_H_ */

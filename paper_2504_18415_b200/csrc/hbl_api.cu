@@ -1,0 +1,318 @@
+// extern "C" entry points of the H-BitLinear library: argument validation,
+// workspace carving and kernel dispatch.  No device memory is allocated here.
+#include <math.h>
+
+#include "hbl_common.cuh"
+
+using namespace hbl;
+
+namespace hbl {
+namespace {
+__device__ int g_status = 0;
+}
+int* device_status_word() {
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess) return nullptr;
+  return static_cast<int*>(p);
+}
+}  // namespace hbl
+
+namespace {
+
+constexpr int kStreamMaxTokens = 64;
+constexpr int kMaxInDim = 32768;
+
+struct ForwardWs {           // byte offsets inside the caller's workspace
+  size_t scale, codesum, zero_region, counters, acc, codes, w_i8, total;
+  size_t zero_words;
+};
+
+ForwardWs carve(int T, int K, int N) {
+  ForwardWs w{};
+  size_t off = 0;
+  w.scale = off;   off = align_up(off + sizeof(float) * (size_t)T, 256);
+  w.codesum = off; off = align_up(off + sizeof(int32_t) * (size_t)T, 256);
+  const int ts = T < kStreamMaxTokens ? T : kStreamMaxTokens;
+  w.zero_region = off;
+  w.counters = off; off += sizeof(int) * align_up(gemm_stream_counter_words(N), 4);
+  w.acc = off;      off += sizeof(int32_t) * gemm_stream_acc_words(ts, N);
+  w.zero_words = (off - w.zero_region) / 4;
+  off = align_up(off, 1024);
+  w.codes = off;   off = align_up(off + (size_t)T * K, 1024);
+  w.w_i8 = off;    off = align_up(off + (size_t)N * K, 1024);
+  w.total = off;
+  return w;
+}
+
+int check_dims(int tokens, int in_dim, int out_dim) {
+  if (tokens < 0 || in_dim <= 0 || out_dim <= 0) return HBL_ERR_SHAPE;
+  if (in_dim % 128 != 0 || out_dim % 16 != 0) return HBL_ERR_SHAPE;
+  if (in_dim > kMaxInDim) return HBL_ERR_TOO_LARGE;
+  return HBL_OK;
+}
+
+int check_quant_args(int x_dtype, int in_dim, int bits, int use_hadamard, float eps) {
+  if (x_dtype != HBL_F32 && x_dtype != HBL_BF16) return HBL_ERR_FORMAT;
+  if (bits != 4 && bits != 8) return HBL_ERR_BITS;
+  if (!(eps > 0.0f) || !isfinite(eps)) return HBL_ERR_EPS;
+  if (use_hadamard && !is_pow2(in_dim)) return HBL_ERR_NOT_POW2;
+  return HBL_OK;
+}
+
+int resolve_path(int path, int tokens) {
+  if (path == HBL_PATH_AUTO) return tokens <= kStreamMaxTokens ? HBL_PATH_STREAM : HBL_PATH_TENSOR;
+  if (path == HBL_PATH_STREAM) return tokens <= kStreamMaxTokens ? HBL_PATH_STREAM : -1;
+  if (path == HBL_PATH_TENSOR) return HBL_PATH_TENSOR;
+  return -2;
+}
+
+// quantized activations -> one projection.  Exactly one of y / acc_out set.
+int run_gemm(int path, const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
+             const void* W_packed, int N, const float* alpha, void* y, int32_t* acc_out, int32_t* acc_ws,
+             int* counters, int8_t* w_i8, cudaStream_t s) {
+  if (path == HBL_PATH_STREAM)
+    return launch_gemm_stream(codes, scale, codesum, T, K, W_packed, N, alpha, static_cast<__nv_bfloat16*>(y),
+                              acc_out, acc_ws, counters, s);
+  int rc = launch_unpack_weights(W_packed, N, K, w_i8, s);
+  if (rc != HBL_OK) return rc;
+  return launch_gemm_tensor(codes, scale, T, K, w_i8, N, alpha, static_cast<__nv_bfloat16*>(y), acc_out, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* hbl_status_string(int status) {
+  switch (status) {
+    case HBL_OK: return "ok";
+    case HBL_ERR_NULL: return "null pointer";
+    case HBL_ERR_SHAPE: return "unsupported shape";
+    case HBL_ERR_NOT_POW2: return "in_dim must be a power of two for the Hadamard transform";
+    case HBL_ERR_BITS: return "bits must be 4 or 8";
+    case HBL_ERR_ALIGN: return "misaligned pointer";
+    case HBL_ERR_WORKSPACE: return "workspace too small";
+    case HBL_ERR_EPS: return "eps must be positive and finite";
+    case HBL_ERR_CUDA: return "CUDA call failed";
+    case HBL_ERR_TIMEOUT: return "device-side wait timed out";
+    case HBL_ERR_FORMAT: return "unknown dtype or path";
+    case HBL_ERR_TOO_LARGE: return "size beyond the supported maximum";
+    default: return "unknown status";
+  }
+}
+
+size_t hbl_packed_weight_bytes(int out_dim, int in_dim) {
+  if (check_dims(0, in_dim, out_dim) != HBL_OK) return 0;
+  return (size_t)out_dim * in_dim / 4;
+}
+
+size_t hbl_workspace_bytes(int max_tokens, int in_dim, int out_dim) {
+  if (check_dims(max_tokens, in_dim, out_dim) != HBL_OK) return 0;
+  return carve(max_tokens, in_dim, out_dim).total;
+}
+
+size_t hbl_quantize_weights_workspace_bytes(int out_dim, int in_dim) {
+  if (check_dims(0, in_dim, out_dim) != HBL_OK) return 0;
+  return 2048 * sizeof(double);
+}
+
+int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_dim, float eps,
+                         void* W_packed, float* alpha, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+  if (!W_latent || !W_packed || !alpha || !workspace) return HBL_ERR_NULL;
+  int rc = check_dims(0, in_dim, out_dim);
+  if (rc != HBL_OK) return rc;
+  if (w_dtype != HBL_F32 && w_dtype != HBL_BF16) return HBL_ERR_FORMAT;
+  if (!(eps > 0.0f) || !isfinite(eps)) return HBL_ERR_EPS;
+  if (!aligned(W_latent, 16) || !aligned(W_packed, 16) || !aligned(alpha, 4) || !aligned(workspace, 16))
+    return HBL_ERR_ALIGN;
+  if (workspace_bytes < hbl_quantize_weights_workspace_bytes(out_dim, in_dim)) return HBL_ERR_WORKSPACE;
+  return launch_weight_quant(W_latent, w_dtype, out_dim, in_dim, eps, W_packed, alpha, workspace,
+                             static_cast<cudaStream_t>(stream));
+}
+
+int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* W_packed,
+                const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y,
+                void* workspace, size_t workspace_bytes, int path, void* stream) {
+  int rc = check_dims(tokens, in_dim, out_dim);
+  if (rc != HBL_OK) return rc;
+  rc = check_quant_args(x_dtype, in_dim, bits, use_hadamard, eps);
+  if (rc != HBL_OK) return rc;
+  const int p = resolve_path(path, tokens);
+  if (p == -1) return HBL_ERR_TOO_LARGE;
+  if (p < 0) return HBL_ERR_FORMAT;
+  if (tokens == 0) return HBL_OK;
+  if (!x || !W_packed || !alpha || !y || !workspace) return HBL_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(W_packed, 16) || !aligned(y, 16) || !aligned(workspace, 1024) ||
+      !aligned(alpha, 4))
+    return HBL_ERR_ALIGN;
+  const ForwardWs w = carve(tokens, in_dim, out_dim);
+  if (workspace_bytes < w.total) return HBL_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  float* scale = reinterpret_cast<float*>(ws + w.scale);
+  int32_t* codesum = reinterpret_cast<int32_t*>(ws + w.codesum);
+  int8_t* codes = reinterpret_cast<int8_t*>(ws + w.codes);
+  const bool stream_path = (p == HBL_PATH_STREAM);
+  rc = launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale, codesum, nullptr,
+                        stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
+                        stream_path ? w.zero_words : 0, s);
+  if (rc != HBL_OK) return rc;
+  return run_gemm(p, codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha, y, nullptr,
+                  reinterpret_cast<int32_t*>(ws + w.acc), reinterpret_cast<int*>(ws + w.counters),
+                  reinterpret_cast<int8_t*>(ws + w.w_i8), s);
+}
+
+// ---- decoder block: four quantizations, seven projections -------------------------------
+namespace {
+struct BlockWs {
+  size_t scale[4], codesum[4], codes[4], zero_region, counters[7], acc[7], w_i8, total, zero_words;
+};
+BlockWs carve_block(int T, int H, int F) {
+  BlockWs w{};
+  const int in_dims[4] = {H, H, H, F};                       // attn_in, o_in, ffn_in, down_in
+  const int out_dims[7] = {H, H, H, H, F, F, H};             // q k v o up gate down
+  size_t off = 0;
+  for (int i = 0; i < 4; ++i) { w.scale[i] = off; off = align_up(off + 4 * (size_t)T, 256); }
+  for (int i = 0; i < 4; ++i) { w.codesum[i] = off; off = align_up(off + 4 * (size_t)T, 256); }
+  const int ts = T < kStreamMaxTokens ? T : kStreamMaxTokens;
+  w.zero_region = off;
+  for (int i = 0; i < 7; ++i) {
+    w.counters[i] = off; off += sizeof(int) * align_up(gemm_stream_counter_words(out_dims[i]), 4);
+    w.acc[i] = off;      off += sizeof(int32_t) * gemm_stream_acc_words(ts, out_dims[i]);
+  }
+  w.zero_words = (off - w.zero_region) / 4;
+  off = align_up(off, 1024);
+  for (int i = 0; i < 4; ++i) { w.codes[i] = off; off = align_up(off + (size_t)T * in_dims[i], 1024); }
+  w.w_i8 = off; off = align_up(off + (size_t)F * H, 1024);   // largest weight: F x H
+  w.total = off;
+  return w;
+}
+}  // namespace
+
+size_t hbl_block_workspace_bytes(int max_tokens, int hidden, int ffn) {
+  if (check_dims(max_tokens, hidden, hidden) != HBL_OK || check_dims(max_tokens, ffn, ffn) != HBL_OK) return 0;
+  return carve_block(max_tokens, hidden, ffn).total;
+}
+
+int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_bytes, int path, void* stream) {
+  if (!b) return HBL_ERR_NULL;
+  const int T = b->tokens, H = b->hidden, F = b->ffn;
+  int rc = check_dims(T, H, H);
+  if (rc != HBL_OK) return rc;
+  rc = check_dims(T, F, F);
+  if (rc != HBL_OK) return rc;
+  rc = check_quant_args(b->x_dtype, H, b->bits, 1, b->eps);
+  if (rc != HBL_OK) return rc;
+  if (!is_pow2(F)) return HBL_ERR_NOT_POW2;
+  const int p = resolve_path(path, T);
+  if (p == -1) return HBL_ERR_TOO_LARGE;
+  if (p < 0) return HBL_ERR_FORMAT;
+  if (T == 0) return HBL_OK;
+  const void* xs[4] = {b->x_attn_in, b->x_o_in, b->x_ffn_in, b->x_down_in};
+  const void* Ws[7] = {b->Wq, b->Wk, b->Wv, b->Wo, b->Wup, b->Wgate, b->Wdown};
+  void* ys[7] = {b->yq, b->yk, b->yv, b->yo, b->yup, b->ygate, b->ydown};
+  for (int i = 0; i < 4; ++i) {
+    if (!xs[i]) return HBL_ERR_NULL;
+    if (!aligned(xs[i], 16)) return HBL_ERR_ALIGN;
+  }
+  for (int i = 0; i < 7; ++i) {
+    if (!Ws[i] || !ys[i]) return HBL_ERR_NULL;
+    if (!aligned(Ws[i], 16) || !aligned(ys[i], 16)) return HBL_ERR_ALIGN;
+  }
+  if (!b->alpha7 || !workspace) return HBL_ERR_NULL;
+  if (!aligned(workspace, 1024)) return HBL_ERR_ALIGN;
+  const BlockWs w = carve_block(T, H, F);
+  if (workspace_bytes < w.total) return HBL_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  const int in_dims[4] = {H, H, H, F};
+  const int had[4] = {0, 1, 0, 1};
+  const bool stream_path = (p == HBL_PATH_STREAM);
+  for (int i = 0; i < 4; ++i) {
+    rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
+                          reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
+                          reinterpret_cast<int32_t*>(ws + w.codesum[i]), nullptr,
+                          (stream_path && i == 0) ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
+                          (stream_path && i == 0) ? w.zero_words : 0, s);
+    if (rc != HBL_OK) return rc;
+  }
+  const int src[7] = {0, 0, 0, 1, 2, 2, 3};                  // which quantized input feeds each projection
+  const int out_dims[7] = {H, H, H, H, F, F, H};
+  for (int i = 0; i < 7; ++i) {
+    const int xi = src[i];
+    rc = run_gemm(p, reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]),
+                  reinterpret_cast<int32_t*>(ws + w.codesum[xi]), T, in_dims[xi], Ws[i], out_dims[i],
+                  b->alpha7 + i, ys[i], nullptr, reinterpret_cast<int32_t*>(ws + w.acc[i]),
+                  reinterpret_cast<int*>(ws + w.counters[i]), reinterpret_cast<int8_t*>(ws + w.w_i8), s);
+    if (rc != HBL_OK) return rc;
+  }
+  return HBL_OK;
+}
+
+int hbl_check_status(void* stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return HBL_ERR_CUDA;
+  int* word = device_status_word();
+  if (word == nullptr) return HBL_ERR_CUDA;
+  int st = 0;
+  if (cudaMemcpy(&st, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return HBL_ERR_CUDA;
+  if (st != 0 && cudaMemset(word, 0, sizeof(int)) != cudaSuccess) return HBL_ERR_CUDA;
+  return st;
+}
+
+int hbl_hadamard_f32(const void* x, int x_dtype, int tokens, int in_dim, float* xr_out, void* stream) {
+  int rc = check_dims(tokens, in_dim, 16);
+  if (rc != HBL_OK) return rc;
+  if (x_dtype != HBL_F32 && x_dtype != HBL_BF16) return HBL_ERR_FORMAT;
+  if (!is_pow2(in_dim)) return HBL_ERR_NOT_POW2;
+  if (tokens == 0) return HBL_OK;
+  if (!x || !xr_out) return HBL_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(xr_out, 16)) return HBL_ERR_ALIGN;
+  return launch_act_quant(x, x_dtype, tokens, in_dim, 4, 1, 1.0f, nullptr, nullptr, nullptr, xr_out, nullptr, 0,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int hbl_quantize_act(const void* x, int x_dtype, int tokens, int in_dim, int bits, int use_hadamard,
+                     float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out, void* stream) {
+  int rc = check_dims(tokens, in_dim, 16);
+  if (rc != HBL_OK) return rc;
+  rc = check_quant_args(x_dtype, in_dim, bits, use_hadamard, eps);
+  if (rc != HBL_OK) return rc;
+  if (tokens == 0) return HBL_OK;
+  if (!x || !codes_out || !scale_out) return HBL_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(codes_out, 16) || !aligned(scale_out, 4)) return HBL_ERR_ALIGN;
+  return launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes_out, scale_out, codesum_out,
+                          nullptr, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in_dim, const void* W_packed,
+                 int out_dim, int32_t* acc_out, void* workspace, size_t workspace_bytes, int path, void* stream) {
+  int rc = check_dims(tokens, in_dim, out_dim);
+  if (rc != HBL_OK) return rc;
+  const int p = resolve_path(path, tokens);
+  if (p == -1) return HBL_ERR_TOO_LARGE;
+  if (p < 0) return HBL_ERR_FORMAT;
+  if (tokens == 0) return HBL_OK;
+  if (!codes || !W_packed || !acc_out || !workspace) return HBL_ERR_NULL;
+  if (p == HBL_PATH_STREAM && !codesum) return HBL_ERR_NULL;
+  if (!aligned(codes, 16) || !aligned(W_packed, 16) || !aligned(acc_out, 16) || !aligned(workspace, 1024))
+    return HBL_ERR_ALIGN;
+  const ForwardWs w = carve(tokens, in_dim, out_dim);
+  if (workspace_bytes < w.total) return HBL_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  if (p == HBL_PATH_STREAM) HBL_CUDA_OK(cudaMemsetAsync(ws + w.zero_region, 0, w.zero_words * 4, s));
+  return run_gemm(p, codes, nullptr, codesum, tokens, in_dim, W_packed, out_dim, nullptr, nullptr, acc_out,
+                  reinterpret_cast<int32_t*>(ws + w.acc), reinterpret_cast<int*>(ws + w.counters),
+                  reinterpret_cast<int8_t*>(ws + w.w_i8), s);
+}
+
+int hbl_unpack_weights(const void* W_packed, int out_dim, int in_dim, int8_t* w_out, void* stream) {
+  int rc = check_dims(0, in_dim, out_dim);
+  if (rc != HBL_OK) return rc;
+  if (!W_packed || !w_out) return HBL_ERR_NULL;
+  if (!aligned(W_packed, 16) || !aligned(w_out, 16)) return HBL_ERR_ALIGN;
+  return launch_unpack_weights(W_packed, out_dim, in_dim, w_out, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

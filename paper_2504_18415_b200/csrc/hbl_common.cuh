@@ -1,0 +1,54 @@
+// Shared declarations of the H-BitLinear CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hbl.h"
+
+namespace hbl {
+
+// ---- device status word (first error wins) --------------------------------
+// Device address of the library's status word on the current device (host call;
+// NULL if the address cannot be obtained).  Kernels receive it as a parameter.
+int* device_status_word();
+__device__ __forceinline__ void report_device_error(int* status, int code) { atomicCAS(status, 0, code); }
+
+// ---- small helpers ----------------------------------------------------------
+__host__ __device__ constexpr int ilog2(unsigned v) { return v <= 1 ? 0 : 1 + ilog2(v >> 1); }
+inline bool is_pow2(long v) { return v > 0 && (v & (v - 1)) == 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+#define HBL_CUDA_OK(expr)                         \
+  do {                                            \
+    cudaError_t _e = (expr);                      \
+    if (_e != cudaSuccess) return HBL_ERR_CUDA;   \
+  } while (0)
+
+// ---- kernel launchers (one per .cu file) -------------------------------------
+// Activation side: Eq. 3-6.
+int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use_hadamard, float eps,
+                     int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
+                     int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s);
+// Weight side: Eq. 1-2 and the 2-bit format.
+int launch_weight_quant(const void* W, int w_dtype, int N, int K, float eps, void* packed, float* alpha,
+                        void* ws, cudaStream_t s);
+int launch_unpack_weights(const void* packed, int N, int K, int8_t* out, cudaStream_t s);
+// Contraction + epilogue.  Exactly one of y / acc_out is written.
+struct GemmSegment {          // one weight tensor of a (possibly fused) projection
+  const void* W;              // packed (stream path) or int8 row-major (tensor path)
+  const float* alpha;         // device, one float (ignored when acc_out is set)
+  void* y;                    // bf16 [T, N]
+  int N;
+};
+int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
+                       const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
+                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s);
+int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
+                       const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s);
+size_t gemm_stream_acc_words(int T, int N);       // int32 words of split-K scratch (0 if none)
+size_t gemm_stream_counter_words(int N);
+
+}  // namespace hbl

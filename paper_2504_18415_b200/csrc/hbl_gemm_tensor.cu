@@ -1,0 +1,338 @@
+// Large-batch contraction of H-BitLinear (Eq. 7) on the 5th-generation tensor
+// cores: tcgen05.mma kind::i8 (int8 x int8 -> int32) with the accumulators in
+// tensor memory, operands staged in shared memory by TMA, and the epilogue
+// (alpha * s_t rescale, one rounding to bf16) reading the accumulators back with
+// tcgen05.ld.
+//
+//   D[128 tokens, 256 weight rows] += A[128, 32] * B[256, 32]^T   per instruction
+//
+// Persistent, warp-specialised, one CTA per SM:
+//   warp 0      TMA producer: 4-stage ring of (A 128x128 B, B 256x128 B) tiles, 128-byte swizzle
+//   warp 1      allocates the 512 TMEM columns, one lane issues the MMAs and commits
+//   warps 2..5  epilogue: each owns the TMEM lane quadrant (warp & 3)
+// Two 256-column accumulators alternate so that the epilogue of tile i overlaps
+// the main loop of tile i+1.
+//
+// Every wait is bounded: when a barrier does not flip within ~2 s the waiting
+// thread records HBL_ERR_TIMEOUT in the status word and raises a CTA-wide abort
+// flag that all roles poll; the CTA then drains, frees its tensor memory and
+// returns.  No TMA multicast is used anywhere.
+#include <cuda.h>
+
+#include "hbl_common.cuh"
+
+namespace hbl {
+namespace {
+
+constexpr int BM = 128;              // tokens per tile (MMA M, TMEM lanes)
+constexpr int BN = 256;              // weight rows per tile (MMA N, TMEM columns)
+constexpr int BK = 128;              // bytes (= int8 elements) of K per stage: one swizzle atom
+constexpr int UMMA_K = 32;           // K of one kind::i8 instruction
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK;     // 16 KiB
+constexpr int B_BYTES = BN * BK;     // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024;   // + alignment slack
+
+// Instruction descriptor (32 bit): D format s32 (2) at bits [4,6); A and B format
+// signed 8-bit (1) at [7,10) and [10,13); both K-major (bits 15, 16 = 0);
+// N >> 3 at [17,23); M >> 4 at [24,29).
+constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                           ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// Shared-memory matrix descriptor, K-major operand in the 128-byte swizzle:
+// start address >> 4 at [0,14); leading byte offset (unused for swizzled K-major) = 1 at [16,30);
+// stride byte offset = 1024 B between 8-row groups, >> 4, at [32,46); version 1 at [46,48);
+// layout type 2 (128-byte swizzle) at [61,64).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when aborted (by this thread's timeout or another role's).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  uint32_t polls = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++polls & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > 2000000000ull) {
+        report_device_error(status, HBL_ERR_TIMEOUT);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);   // .x = a (low half), .y = b
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                   const float* __restrict__ scale, const float* __restrict__ alpha,
+                   __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out, int T, int N, int K,
+                   int* __restrict__ status) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) uint64_t full_bar[STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ __align__(8) uint64_t tfull_bar[2];
+  __shared__ __align__(8) uint64_t tempty_bar[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+
+  unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (T + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int nkb = K / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tfull_bar[b], 1); mbar_init(&tempty_bar[b], 4); }
+    abort_flag_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                 "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abort_flag, status)) { ok = false; break; }
+          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+          unsigned char* a = tiles + (size_t)s * STAGE_BYTES;
+          tma_load_2d(a, &tmA, &full_bar[s], kb * BK, m0);
+          tma_load_2d(a + A_BYTES, &tmB, &full_bar[s], kb * BK, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tl) {
+        const int b = tl & 1;
+        if (!mbar_wait(&tempty_bar[b], ((tl >> 1) & 1) ^ 1, abort_flag, status)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)b * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&full_bar[s], (it / STAGES) & 1, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(tiles + (size_t)s * STAGE_BYTES);
+          const uint64_t adesc = make_desc(a_addr), bdesc = make_desc(a_addr + A_BYTES);
+#pragma unroll
+          for (int ks = 0; ks < BK / UMMA_K; ++ks)
+            umma_i8(d_tmem, adesc + (uint64_t)(ks * UMMA_K / 16), bdesc + (uint64_t)(ks * UMMA_K / 16),
+                    (kb | ks) != 0);
+          umma_commit(&empty_bar[s]);          // stage reusable once these MMAs have read it
+        }
+        if (ok) umma_commit(&tfull_bar[b]);    // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ------------------------------
+    const int q = warp & 3;                    // TMEM lane quadrant this warp may access
+    const float al = (acc_out == nullptr) ? __ldg(alpha) : 0.f;
+    uint32_t tl = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tl) {
+      const int b = tl & 1;
+      const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+      const bool got = mbar_wait(&tfull_bar[b], (tl >> 1) & 1, abort_flag, status);
+      if (!__all_sync(0xffffffffu, got)) break;      // warp-uniform: tcgen05.ld needs the whole warp
+      tc_fence_after();
+      const int row = m0 + q * 32 + lane;
+      const float f = (acc_out == nullptr && row < T) ? __ldg(scale + row) * al : 0.f;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * 32), r);
+        tmem_ld_wait();
+        const int col = n0 + c * 32;
+        if (row < T) {
+          if (acc_out != nullptr) {
+            int32_t* dst = acc_out + (size_t)row * N + col;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              if (col + i < N) *reinterpret_cast<uint4*>(dst + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+          } else {
+            __nv_bfloat16* dst = y + (size_t)row * N + col;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              if (col + i < N) {
+                uint4 o;
+                o.x = pack_bf16((float)(int)r[i + 0] * f, (float)(int)r[i + 1] * f);
+                o.y = pack_bf16((float)(int)r[i + 2] * f, (float)(int)r[i + 3] * f);
+                o.z = pack_bf16((float)(int)r[i + 4] * f, (float)(int)r[i + 5] * f);
+                o.w = pack_bf16((float)(int)r[i + 6] * f, (float)(int)r[i + 7] * f);
+                *reinterpret_cast<uint4*>(dst + i) = o;
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty_bar[b]);
+    }
+  }
+
+  // ------------------------------ teardown ------------------------------
+  __syncwarp();
+  if (*abort_flag) {
+    // give copies that are still in flight time to land before the CTA's shared memory goes away
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---- host side: tensor maps through the driver entry point (no libcuda link) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// int8 matrix [rows, K] row-major, box = box_rows x 128 bytes, 128-byte swizzle, zero fill.
+int make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return HBL_ERR_CUDA;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? HBL_OK : HBL_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
+                       const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s) {
+  if (T <= 0) return HBL_OK;
+  CUtensorMap tmA, tmB;
+  int rc = make_map(&tmA, codes, T, K, BM);
+  if (rc != HBL_OK) return rc;
+  rc = make_map(&tmB, W_i8, N, K, BN);
+  if (rc != HBL_OK) return rc;
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    HBL_CUDA_OK(cudaGetDevice(&dev));
+    HBL_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+    HBL_CUDA_OK(cudaFuncSetAttribute(gemm_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  }
+  int* status = device_status_word();
+  if (status == nullptr) return HBL_ERR_CUDA;
+  const int n_tiles = ((T + BM - 1) / BM) * ((N + BN - 1) / BN);
+  const int grid = n_tiles < n_sm ? n_tiles : n_sm;
+  gemm_tensor_kernel<<<grid, THREADS, SMEM_BYTES, s>>>(tmA, tmB, scale, alpha, y, acc_out, T, N, K, status);
+  HBL_CUDA_OK(cudaGetLastError());
+  return HBL_OK;
+}
+
+}  // namespace hbl

@@ -1,0 +1,105 @@
+"""GPU parity: transform (Eq. 3-4) and activation quantizers (Eq. 5-6) vs the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hbl_oracle as orc
+from paper_2504_18415_b200 import hbl, workloads as wl
+from parity_utils import EPS, check_codes, to_dev
+
+pytestmark = pytest.mark.gpu
+
+ALL_K = [128, 256, 512, 1024, 2048, 4096, 8192, 16384, 32768]
+
+
+def make_x(K, T, seed, kind="attn_out", dtype="bf16"):
+    return wl.rows(kind, seed, 1, K, 0, T, dtype)
+
+
+@pytest.mark.parametrize("K", ALL_K)
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_hadamard_matches_oracle(K, dtype):
+    T = 37 if K <= 8192 else 9           # ragged against every tokens-per-CTA grouping
+    x = make_x(K, T, 100 + K, dtype=dtype)
+    got = hbl.hbl_hadamard_f32(to_dev(x, dtype)).cpu().numpy().astype(np.float64)
+    want = orc.hadamard(x)
+    tol = 1e-5 * np.abs(want).max(axis=1, keepdims=True)
+    assert np.all(np.abs(got - want) <= tol), float((np.abs(got - want) / tol).max())
+
+
+def test_hadamard_unit_vectors_and_involution():
+    K = 4096
+    x = np.zeros((4, K), np.float32)
+    x[0, 0] = 1; x[1, 1] = 1; x[2, K - 1] = 1; x[3, :] = 1
+    got = hbl.hbl_hadamard_f32(to_dev(x, "f32")).cpu().numpy()
+    idx = np.arange(K)
+    s = 1 / 64.0
+    assert np.array_equal(got[0], np.full(K, s, np.float32))
+    assert np.array_equal(got[1], np.where(idx & 1, -s, s).astype(np.float32))
+    par = np.array([bin(i).count("1") & 1 for i in idx])
+    assert np.array_equal(got[2], np.where(par, -s, s).astype(np.float32))
+    assert got[3, 0] == 64.0 and np.all(got[3, 1:] == 0)
+    y = wl.rows("gauss", 1, 1, K, 0, 8, "f32")
+    back = hbl.hbl_hadamard_f32(hbl.hbl_hadamard_f32(to_dev(y, "f32"))).cpu().numpy()
+    assert np.allclose(back, y, atol=1e-5 * np.abs(y).max())
+
+
+@pytest.mark.parametrize("K", ALL_K)
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("had", [True, False])
+def test_quantize_act_matches_oracle(K, bits, had):
+    T = 67 if K <= 8192 else 11
+    kind = "ffn_mid" if K >= 8192 else "attn_out"
+    x = make_x(K, T, 7 * K + bits, kind)
+    codes, scale, csum = hbl.hbl_quantize_act(to_dev(x, "bf16"), bits, had, EPS)
+    xr = orc.hadamard(x) if had else x.astype(np.float64)
+    q, v, s, st = orc.act_quant(xr, bits, EPS, 32)
+    cg = codes.cpu().numpy()
+    check_codes(cg, q, v)
+    assert np.allclose(scale.cpu().numpy(), s, rtol=2e-6, atol=0)
+    assert np.array_equal(csum.cpu().numpy(), cg.astype(np.int64).sum(1))
+    lo, hi = (-128, 127) if bits == 8 else (-8, 7)
+    assert cg.min() >= lo and cg.max() <= hi
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_quantize_act_without_transform_is_bit_exact(bits):
+    """No transform: the statistic is exact in fp32, so both sides take identical decisions
+    (INT8: max is exact; INT4: the fp32 sum order may differ by an ulp, hence the tolerance rule)."""
+    K, T = 4096, 130
+    x = wl.rows("gauss", 4, 1, K, 0, T, "bf16")
+    codes, scale, _ = hbl.hbl_quantize_act(to_dev(x, "bf16"), bits, False, EPS)
+    q, v, s, st = orc.act_quant(x.astype(np.float64), bits, EPS, 32)
+    if bits == 8:
+        assert np.array_equal(codes.cpu().numpy(), q)
+        assert np.array_equal(scale.cpu().numpy(), s.astype(np.float32))
+    else:
+        check_codes(codes.cpu().numpy(), q, v)
+
+
+def test_quantize_act_generic_width_and_fp32_input():
+    K, T = 384, 19                       # not a power of two: plain BitLinear input only
+    x = wl.rows("gauss", 9, 1, K, 0, T, "f32")
+    for bits in (4, 8):
+        codes, scale, csum = hbl.hbl_quantize_act(to_dev(x, "f32"), bits, False, EPS)
+        q, v, s, st = orc.act_quant(x.astype(np.float64), bits, EPS, 32)
+        check_codes(codes.cpu().numpy(), q, v)
+        assert np.allclose(scale.cpu().numpy(), s, rtol=2e-6)
+        assert np.array_equal(csum.cpu().numpy(), codes.cpu().numpy().astype(np.int64).sum(1))
+    with pytest.raises(hbl.HblError):
+        hbl.hbl_quantize_act(to_dev(x, "f32"), 4, True, EPS)
+
+
+def test_degenerate_tokens():
+    K = 2048
+    x = np.zeros((3, K), np.float32)
+    x[1, 5] = 3.0                         # a single spike: the transform spreads it evenly
+    x[2, :] = -2.0                        # constant: the transform concentrates it in index 0
+    for bits in (4, 8):
+        codes, scale, csum = hbl.hbl_quantize_act(to_dev(x, "bf16"), bits, True, EPS)
+        c = codes.cpu().numpy(); sc = scale.cpu().numpy()
+        assert np.all(c[0] == 0) and sc[0] == 0.0
+        q, v, s, st = orc.act_quant(orc.hadamard(x), bits, EPS, 32)
+        check_codes(c, q, v)
+        assert np.all(np.isfinite(sc))
+    assert hbl.hbl_quantize_act(torch.empty((0, K), dtype=torch.bfloat16, device="cuda"), 4, True, EPS)[0].shape[0] == 0

@@ -1,0 +1,107 @@
+"""GPU parity: the whole layer (Eq. 3-7) through hbl_forward / hbl_block_forward vs the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hbl_oracle as orc
+from paper_2504_18415_b200 import hbl, workloads as wl
+from parity_utils import EPS, check_codes, check_y, oracle_layer, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def run_layer(x, W, bits, had, dtype, path):
+    Wd = torch.from_numpy(W).cuda()
+    packed, alpha = hbl.hbl_quantize_weights(Wd, EPS)
+    y = hbl.hbl_forward(to_dev(x, dtype), packed, alpha, W.shape[0], bits, had, EPS, path=path)
+    assert hbl.hbl_check_status() == 0
+    return y, packed, alpha
+
+
+def test_config1_full_oracle_check():
+    cfg = wl.CONFIG1
+    x, W = cfg.x(0, 64), cfg.w_latent()
+    o = oracle_layer(x, W, 4, True)
+    for path in (hbl.PATH_AUTO, hbl.PATH_STREAM, hbl.PATH_TENSOR):
+        y, packed, alpha = run_layer(x, W, 4, True, "f32", path)
+        assert alpha.item() == o["alpha"]
+        assert np.array_equal(hbl.hbl_unpack_weights(packed, 512, 512).cpu().numpy(), o["wt"])
+        check_y(y, o["y64"])
+    codes, scale, csum = hbl.hbl_quantize_act(to_dev(x, "f32"), 4, True, EPS)
+    nbad = check_codes(codes.cpu().numpy(), o["q"], o["v"])
+    if nbad == 0:      # identical codes => identical accumulators => y differs by the bf16 rounding only
+        yf = y.float().cpu().numpy()
+        yo = orc.bf16_bits_to_f32(o["y_bits"])
+        assert np.all(np.abs(yf - yo) <= np.abs(yo) * 2.0 ** -7 + 1e-30)
+
+
+@pytest.mark.parametrize("T", [1, 5, 16, 40, 64, 65, 200, 513])
+@pytest.mark.parametrize("bits,had", [(4, True), (8, True), (4, False), (8, False)])
+def test_layer_small_shapes(T, bits, had):
+    K, N = 1024, 784                      # N ragged against both kernels' tiles
+    x = wl.rows("attn_out", 21, 1, K, 0, T, "bf16")
+    W = wl.rows("latent", 21, 2, K, 0, N, "f32")
+    o = oracle_layer(x, W, bits, had)
+    y, _, _ = run_layer(x, W, bits, had, "bf16", hbl.PATH_AUTO)
+    check_y(y, o["y64"])
+
+
+def test_hand_worked_layer_value_scaled_up():
+    """The hand-worked 4-wide example embedded in a 128-wide layer (zero padding keeps
+    beta*K and the codes' pattern predictable): checks sign, operand order and scale."""
+    K, N = 128, 16
+    x = np.zeros((1, K), np.float32); x[0, :4] = [1, 2, 3, 4]
+    W = np.zeros((N, K), np.float32)
+    W[0, :4] = [0.3, -0.1, 0.05, -0.4]; W[1, :4] = [-0.02, 0.5, 0.2, -0.2]
+    o = oracle_layer(x, W, 4, False)
+    y, _, _ = run_layer(x, W, 4, False, "f32", hbl.PATH_AUTO)
+    check_y(y, o["y64"])
+    assert np.array_equal(y.float().cpu().numpy(), orc.bf16_bits_to_f32(o["y_bits"]))
+
+
+def test_token_permutation_and_scaling_properties():
+    K, N, T = 2048, 2048, 16
+    x = wl.CONFIG2.x(0, T)
+    W = wl.CONFIG2.w_latent()
+    packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), EPS)
+    xd = to_dev(x, "bf16")
+    y = hbl.hbl_forward(xd, packed, alpha, N, 4, True, EPS)
+    perm = torch.randperm(T, generator=torch.Generator().manual_seed(0)).cuda()
+    yp = hbl.hbl_forward(xd[perm].contiguous(), packed, alpha, N, 4, True, EPS)
+    assert torch.equal(yp, y[perm])
+    y4 = hbl.hbl_forward((xd * 4).contiguous(), packed, alpha, N, 4, True, EPS)
+    # eps does not scale with the token, so a few codes next to a rounding boundary may move:
+    # compare against the row's rms like the parity bar does.
+    ref = 4 * y.float()
+    tol = 2e-2 * torch.maximum(ref.abs(), ref.pow(2).mean(1, keepdim=True).sqrt())
+    assert torch.all((y4.float() - ref).abs() <= tol)
+    # one token alone gives the same row as inside a batch, on either kernel
+    y1 = hbl.hbl_forward(xd[3:4].contiguous(), packed, alpha, N, 4, True, EPS, path=hbl.PATH_TENSOR)
+    assert torch.equal(y1[0], y[3])
+
+
+def test_block_forward_small():
+    H, F, T = 512, 2048, 24
+    seed = 31
+    ins = {"attn_in": wl.rows("gauss", seed, 10, H, 0, T, "bf16"), "o_in": wl.rows("attn_out", seed, 11, H, 0, T, "bf16"),
+           "ffn_in": wl.rows("gauss", seed, 12, H, 0, T, "bf16"), "down_in": wl.rows("ffn_mid", seed, 13, F, 0, T, "bf16")}
+    shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "up": (F, H), "gate": (F, H), "down": (H, F)}
+    src = {"q": "attn_in", "k": "attn_in", "v": "attn_in", "o": "o_in", "up": "ffn_in", "gate": "ffn_in", "down": "down_in"}
+    Wl = {n: wl.rows("latent", seed, 20 + i, s[1], 0, s[0], "f32") for i, (n, s) in enumerate(shapes.items())}
+    packed, alphas = {}, []
+    for n in shapes:
+        p, a = hbl.hbl_quantize_weights(torch.from_numpy(Wl[n]).cuda(), EPS)
+        packed[n] = p; alphas.append(a)
+    alpha7 = torch.cat(alphas)
+    for path, Tn in ((hbl.PATH_AUTO, T), (hbl.PATH_TENSOR, T)):
+        outs = hbl.hbl_block_forward({k: to_dev(v, "bf16") for k, v in ins.items()}, packed, alpha7, H, F, 4, EPS, path=path)
+        assert hbl.hbl_check_status() == 0
+        for n in shapes:
+            o = oracle_layer(ins[src[n]], Wl[n], 4, n in ("o", "down"))
+            check_y(outs[n], o["y64"])
+
+
+def test_zero_tokens_is_a_noop():
+    packed, alpha = hbl.hbl_quantize_weights(torch.zeros((16, 128), device="cuda"), EPS)
+    y = hbl.hbl_forward(torch.empty((0, 128), dtype=torch.bfloat16, device="cuda"), packed, alpha, 16, 4, True)
+    assert y.shape == (0, 16)
