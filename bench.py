@@ -1,0 +1,498 @@
+#!/usr/bin/env python
+"""Benchmark of the H-BitLinear forward path (one JSON line on stdout).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--sweep none|quick|full]
+
+A "step" is one hbl_forward call (transform + quantize + contraction + rescale)
+over one batch of the headline workload: the W_down-shaped H-BitLinear layer of
+the 1.3B model (in 8192 -> out 2048, INT4 activations, Hadamard on) at 16384
+tokens.  `value` is tokens/s with inputs resident in HBM; `e2e` is the same
+call fed from pinned host memory with the copies inside the timed region.
+The other workload points (small-batch weight streaming, the INT8 setting, the
+7B decoder block) are reported under "points".
+
+With N > 1 (torchrun, one rank per GPU) every rank runs an independent replica
+of the same step (tokens are independent: no collective on the data path); the
+time is the max over ranks and `value` the sum of tokens over ranks.
+
+`--impl reference` times the CPU oracle (the only reference implementation
+there is) on a bounded token sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+EPS = 1e-5
+L2_BYTES = 126 * 1024 * 1024
+RING_BYTES = 4 * L2_BYTES            # ring of distinct input sets so that every call is L2-cold
+NOMINAL_INT8_TOPS = 4500.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"]))}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            f = [c.strip() for c in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [c for c, p in zip(sm, power) if p > 0.5 * max(power)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+# ----------------------------------------------------------------------------- workload helpers
+def alg_bytes(T, K, N, x_bytes=2):
+    """Algorithmic HBM bytes of one layer call: activations in, packed weights, bf16 out."""
+    return T * K * x_bytes + N * K // 4 + 2 * T * N + 4
+
+
+def device_x(cfg_kind, seed, tid, K, T, dtype, torch, max_host_rows=4096):
+    """Activations per the workload recipe; beyond max_host_rows the seeded block is tiled."""
+    from paper_2504_18415_b200 import workloads as wl
+    rows = min(T, max_host_rows)
+    x = torch.from_numpy(wl.rows(cfg_kind, seed, tid, K, 0, rows, dtype)).cuda()
+    if dtype == "bf16":
+        x = x.to(torch.bfloat16)
+    if rows < T:
+        x = x.repeat((T + rows - 1) // rows, 1)[:T].contiguous()
+    return x
+
+
+def device_weights(N, K, seed, torch, hbl):
+    """Latent N(0, 0.02^2) weights drawn on the device (seeded), ternarised by the library."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    W = torch.randn((N, K), generator=g, device="cuda", dtype=torch.float32) * 0.02
+    packed, alpha = hbl.hbl_quantize_weights(W, EPS)
+    del W
+    return packed, alpha
+
+
+def time_loop(fn, iters, warmup, torch):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def layer_point(name, kind, seed, K, N, bits, had, T, torch, hbl, peaks, iters=None):
+    """One single-layer workload point, L2-cold (ring of distinct input sets), returns a dict."""
+    per_call = alg_bytes(T, K, N) + T * K          # + the int8 codes round trip (implementation traffic)
+    ring = max(2, min(64, -(-RING_BYTES // per_call)))
+    if T * K * 2 > 2 * L2_BYTES:
+        ring = 2
+    xs, ws, ys = [], [], []
+    x0 = device_x(kind, seed, 1, K, T, "bf16", torch)
+    for r in range(ring):
+        xs.append(torch.roll(x0, shifts=r, dims=0) if r else x0)
+        ws.append(device_weights(N, K, 1000 * seed + r, torch, hbl))
+        ys.append(torch.empty((T, N), dtype=torch.bfloat16, device="cuda"))
+    wsb = hbl.hbl_workspace_bytes(T, K, N)
+    work = hbl.new_workspace(wsb)
+    path = hbl.PATH_AUTO
+    state = {"i": 0}
+
+    def call():
+        r = state["i"] % ring
+        state["i"] += 1
+        hbl.hbl_forward(xs[r], ws[r][0], ws[r][1], N, bits, had, EPS, y=ys[r], workspace=work, path=path)
+
+    small = T <= 64
+    if small:
+        # launch-latency hiding: one CUDA graph of `ring` back-to-back calls
+        for _ in range(2):
+            for _ in range(ring):
+                call()
+        torch.cuda.synchronize()
+        state["i"] = 0
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(ring):
+                call()
+        reps = iters or 20
+        ms = time_loop(g.replay, reps, 3, torch) / ring
+    else:
+        flops = 2.0 * T * K * N
+        est_ms = max(0.02, flops / 2.0e15 * 1e3)
+        n_it = iters or int(max(5, min(50, 200.0 / est_ms)))
+        ms = time_loop(call, n_it, 3, torch)
+    st = hbl.hbl_check_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} in {name}")
+    tops = 2.0 * T * K * N / (ms * 1e-3) / 1e12
+    gbs = alg_bytes(T, K, N) / (ms * 1e-3) / 1e9
+    out = {"point": name, "tokens": T, "in": K, "out": N, "bits": bits, "hadamard": bool(had),
+           "ms": round(ms, 5), "tokens_per_s": round(T / (ms * 1e-3), 1), "tops": round(tops, 2),
+           "alg_gbs": round(gbs, 1), "ring": ring, "graph": small}
+    if small or tops < 100:
+        out["bound"] = "hbm"
+        out["frac"] = round(gbs / peaks["hbm_gbs"], 4)
+    else:
+        out["bound"] = "tensor"
+        out["frac"] = round(tops / (2 * peaks["bf16_tflops"]), 4)
+        out["frac_of_nominal_int8"] = round(tops / NOMINAL_INT8_TOPS, 4)
+    del xs, ws, ys, work
+    torch.cuda.empty_cache()
+    return out
+
+
+def block_point(T, torch, hbl, peaks, iters=None):
+    """7B-shaped decoder-block projection sweep point (config 5)."""
+    from paper_2504_18415_b200 import workloads as wl
+    cfg = wl.CONFIG5
+    H, F = cfg.hidden, cfg.ffn
+    shapes = cfg.weight_shapes()
+    w_bytes = sum(n * k // 4 for n, k in shapes.values())
+    per_call = w_bytes + T * (3 * H + F) * 2 + 2 * T * (5 * H + 2 * F)
+    small = T <= 64
+    ring = max(2, min(8, -(-RING_BYTES // per_call))) if T < 4096 else 1
+    ins = {"attn_in": device_x("gauss", cfg.seed, 10, H, T, "bf16", torch),
+           "o_in": device_x("attn_out", cfg.seed, 11, H, T, "bf16", torch),
+           "ffn_in": device_x("gauss", cfg.seed, 12, H, T, "bf16", torch),
+           "down_in": device_x("ffn_mid", cfg.seed, 13, F, T, "bf16", torch)}
+    sets = []
+    for r in range(ring):
+        packed, alphas = {}, []
+        for i, (n, (N, K)) in enumerate(shapes.items()):
+            p, a = device_weights(N, K, 5000 + 10 * r + i, torch, hbl)
+            packed[n] = p
+            alphas.append(a)
+        sets.append((packed, torch.cat(alphas)))
+    dims = {"q": H, "k": H, "v": H, "o": H, "up": F, "gate": F, "down": H}
+    outs = {n: torch.empty((T, d), dtype=torch.bfloat16, device="cuda") for n, d in dims.items()}
+    work = hbl.new_workspace(hbl.hbl_block_workspace_bytes(T, H, F))
+    state = {"i": 0}
+
+    def call():
+        r = state["i"] % ring
+        state["i"] += 1
+        hbl.hbl_block_forward(ins, sets[r][0], sets[r][1], H, F, 4, EPS, outputs=outs, workspace=work)
+
+    if small:
+        for _ in range(2 * ring):
+            call()
+        torch.cuda.synchronize()
+        state["i"] = 0
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(ring):
+                call()
+        ms = time_loop(g.replay, iters or 10, 3, torch) / ring
+    else:
+        flops = 2.0 * T * sum(n * k for n, k in shapes.values())
+        est_ms = flops / 2.0e15 * 1e3
+        ms = time_loop(call, iters or int(max(3, min(30, 300.0 / est_ms))), 2, torch)
+    st = hbl.hbl_check_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} in block T={T}")
+    ops = 2.0 * T * sum(n * k for n, k in shapes.values())
+    tops = ops / (ms * 1e-3) / 1e12
+    gbs = per_call / (ms * 1e-3) / 1e9
+    out = {"point": "config5_block_7B", "tokens": T, "ms": round(ms, 5), "tokens_per_s": round(T / (ms * 1e-3), 1),
+           "tops": round(tops, 2), "alg_gbs": round(gbs, 1), "ring": ring, "graph": small}
+    if tops < 100 or small:
+        out["bound"] = "hbm"; out["frac"] = round(gbs / peaks["hbm_gbs"], 4)
+    else:
+        out["bound"] = "tensor"; out["frac"] = round(tops / (2 * peaks["bf16_tflops"]), 4)
+        out["frac_of_nominal_int8"] = round(tops / NOMINAL_INT8_TOPS, 4)
+    del ins, sets, outs, work
+    torch.cuda.empty_cache()
+    return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+HEAD = dict(name="config3_Wdown_1p3B", kind="ffn_mid", seed=3, K=8192, N=2048, bits=4, had=True, T=16384)
+
+
+def oracle_rate(target_s=12.0):
+    """Times the oracle as it stands on a bounded token sample of the headline workload."""
+    from oracle import hbl_oracle as orc
+    from paper_2504_18415_b200 import workloads as wl
+    cores = orc.num_threads()
+    cfg = wl.CONFIG3
+    wt, alpha = orc.weight_quant(cfg.w_latent(), EPS, 32)
+    n0 = max(cores, 8)
+    x = cfg.x(0, n0)
+    t0 = time.perf_counter()
+    orc.forward(x, wt, alpha, cfg.bits, True, EPS, 32)
+    dt = time.perf_counter() - t0
+    n = int(max(n0, min(4096, n0 * target_s / max(dt, 1e-3))))
+    n = (n // cores) * cores or cores
+    x = cfg.x(0, n)
+    t0 = time.perf_counter()
+    orc.forward(x, wt, alpha, cfg.bits, True, EPS, 32)
+    dt = time.perf_counter() - t0
+    return {"value": round(n / dt, 2), "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"{n} tokens of {HEAD['name']} (in 8192 -> out 2048, INT4+Hadamard), all outputs, {dt:.1f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import hbl_oracle as orc
+    from paper_2504_18415_b200 import workloads as wl
+    cores = orc.num_threads()
+    cfg = wl.CONFIG3
+    wt, alpha = orc.weight_quant(cfg.w_latent(), EPS, 32)
+    n = max(cores, 16) * 4
+    x = cfg.x(0, n)
+    for _ in range(max(1, min(args.warmup, 3))):
+        orc.forward(x[:cores], wt, alpha, cfg.bits, True, EPS, 32)
+    t0 = time.perf_counter()
+    steps = max(1, min(args.steps, 20))
+    for _ in range(steps):
+        orc.forward(x, wt, alpha, cfg.bits, True, EPS, 32)
+    dt = (time.perf_counter() - t0) / steps
+    val = n / dt
+    sample = f"each step = {n} tokens of {HEAD['name']} through the CPU oracle (all 2048 outputs)"
+    print(json.dumps({
+        "impl": "reference", "metric": "H-BitLinear forward throughput", "value": round(val, 2), "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{HEAD['name']}: in 8192 -> out 2048, INT4 + Hadamard, bf16 activations (SiLU(a)*b with "
+                               f"0.2% outlier channels x40), {HEAD['T']} tokens per step on the GPU arm; bounded sample here"},
+        "cpu_baseline": {"value": round(val, 2), "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(val, 2), "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ----------------------------------------------------------------------------- main (GPU arm)
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", default="quick", choices=["none", "quick", "full"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2504_18415_b200 import hbl, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks, peak_src = load_peaks()
+    W = max(args.warmup, 3)
+    Ksteps = max(args.steps, 1)
+
+    # ---- headline workload: config 3 at T = 16384, full host-generated seeded inputs ----
+    h = HEAD
+    T, K, N = h["T"], h["K"], h["N"]
+    cfg = wl.CONFIG3
+    x_host = torch.from_numpy(cfg.x(0, T)).to(torch.bfloat16)
+    xs = [x_host.cuda(), torch.roll(x_host, 1, 0).cuda()]            # two 268 MB inputs: every step is L2-cold
+    packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(cfg.w_latent()).cuda(), EPS)
+    ys = [torch.empty((T, N), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    work = hbl.new_workspace(hbl.hbl_workspace_bytes(T, K, N))
+
+    def step(i):
+        hbl.hbl_forward(xs[i & 1], packed, alpha, N, h["bits"], h["had"], EPS, y=ys[i & 1], workspace=work)
+
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = hbl.hbl_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    with hbl.KernelTimer(Ksteps, 2) as kt:
+        e0.record()
+        for i in range(Ksteps):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+    launches = hbl.hbl_launch_count() - launches0
+    total_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        total_ms = float(t.item())
+    torch.cuda.synchronize()
+    # keep the GPU busy a little longer so that the clock sampler sees load
+    if rank == 0:
+        t_end = time.time() + 0.6
+        i = 0
+        while time.time() < t_end:
+            step(i); i += 1
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    gemm_ms = statistics.mean(kt.times_ms())
+    st = hbl.hbl_check_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st}")
+    ms_per_step = total_ms / Ksteps
+    value = world * T / (ms_per_step * 1e-3)
+
+    # per-kernel breakdown (outside the timed region)
+    breakdown = {}
+    for kid, name in ((1, "act_quant_kernel"), (3, "unpack_kernel"), (2, "gemm_tensor_kernel")):
+        with hbl.KernelTimer(5, kid) as k2:
+            for i in range(5):
+                step(i)
+        breakdown[name] = round(statistics.mean(k2.times_ms()), 5)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- e2e: same call, host-resident x and y, copies inside the timed region ----
+    xh = x_host.pin_memory()
+    yh = torch.empty((T, N), dtype=torch.bfloat16).pin_memory()
+    for i in range(2):
+        hbl.hbl_forward_host(xh, packed, alpha, N, h["bits"], h["had"], yh, xs[0], ys[0], work)
+    torch.cuda.synchronize()
+    n_e2e = min(Ksteps, 10)
+    t0 = time.perf_counter()
+    for i in range(n_e2e):
+        hbl.hbl_forward_host(xh, packed, alpha, N, h["bits"], h["had"], yh, xs[0], ys[0], work)
+        torch.cuda.synchronize()
+        _ = float(yh[0, 0])                                           # the host reads the step's result
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+    e2e = {"value": round(T / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "h2d_bytes_per_step": T * K * 2,
+           "d2h_bytes_per_step": T * N * 2, "ms_per_step": round(e2e_ms, 3), "steps": n_e2e}
+
+    ops = 2.0 * T * K * N
+    ach = ops / (gemm_ms * 1e-3) / 1e12
+    peak_i8 = 2.0 * peaks["bf16_tflops"]
+    roofline = {"kernel": "gemm_tensor_kernel (tcgen05.mma kind::i8, 128x256x128 tiles)", "bound": "tensor",
+                "achieved": round(ach, 2), "peak": round(peak_i8, 1), "unit": "TFLOP/s", "frac": round(ach / peak_i8, 4),
+                "traffic": None,
+                "note": f"int8 multiply-add = 2 ops; peak = 2 x {peak_src} bf16 burst (nominal int8:bf16 ratio); "
+                        f"of nominal 4500: {ach / NOMINAL_INT8_TOPS:.3f}; kernel avg {gemm_ms * 1e3:.1f} us over {len(kt.times_ms())} launches"}
+    tr = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tr):
+        try:
+            roofline["traffic"] = json.load(open(tr)).get("gemm_tensor_kernel_bytes_per_launch")
+        except Exception:
+            pass
+
+    points = []
+    if args.sweep != "none" and world == 1:
+        del xs, ys, work
+        torch.cuda.empty_cache()
+        full = args.sweep == "full"
+        L = lambda *a, **k: points.append(layer_point(*a, torch=torch, hbl=hbl, peaks=peaks, **k))
+        for T_ in (1, 16, 256, 4096):
+            L("config2_Wo_1p3B", "attn_out", 2, 2048, 2048, 4, True, T_)
+        for T_ in (1, 16, 1024):
+            L("config3_Wdown_1p3B", "ffn_mid", 3, 8192, 2048, 4, True, T_)
+        for N_ in (12288, 32768):
+            for T_ in ((16, 4096, 32768) if full else (16, 4096)):
+                L(f"config4_a8_N{N_}", "gauss", 4, 4096, N_, 8, False, T_)
+        for T_ in ((1, 4, 16, 64, 256, 1024, 4096, 16384, 65536) if full else (1, 16, 256, 4096)):
+            points.append(block_point(T_, torch, hbl, peaks))
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu = oracle_rate()
+
+    out = {
+        "metric": "H-BitLinear forward throughput (tokens/s; TOPS vs INT8 tensor peak and HBM GB/s under roofline/points)",
+        "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": Ksteps, "warmup": W,
+        "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "s8", "data": "synthetic",
+        "config": {"workload": f"{h['name']}: H-BitLinear in 8192 -> out 2048, INT4 activations + Hadamard, "
+                               f"{T} tokens per step, bf16 activations SiLU(a)*b with 0.2% outlier channels x40, "
+                               f"ternary weights from N(0,0.02) latents",
+                   "l2": "two alternating 268 MB input batches (each larger than the 126 MB L2)",
+                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "tops": round(ops / (ms_per_step * 1e-3) / 1e12, 2),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "kernels_ms": breakdown, "roofline": roofline, "cpu_baseline": cpu, "points": points,
+        "peaks": {**peaks, "source": peak_src, "int8_nominal_tops": NOMINAL_INT8_TOPS},
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -114,6 +114,28 @@ size_t hbl_block_workspace_bytes(int max_tokens, int hidden, int ffn);
 int hbl_block_forward(const hbl_block_t* block /* host pointer */, void* workspace,
                       size_t workspace_bytes, int path, void* stream);
 
+/* hbl_forward for callers whose tensors live in HOST memory (pinned for the copies
+ * to be asynchronous): copies x_host -> x_stage, runs the layer, copies y_stage ->
+ * y_host, all enqueued on `stream`.  x_stage / y_stage are DEVICE staging buffers
+ * of tokens*in_dim*sizeof(x) and tokens*out_dim*2 bytes owned by the caller.
+ * No counterpart in the paper beyond Eq. 3-7 themselves. */
+int hbl_forward_host(const void* x_host /* host */, int x_dtype, int tokens, int in_dim,
+                     const void* W_packed, const float* alpha, int out_dim, int bits, int use_hadamard,
+                     float eps, void* y_host /* host */, void* x_stage, void* y_stage,
+                     void* workspace, size_t workspace_bytes, int path, void* stream);
+
+/* Instrumentation (host-side state, not thread-safe).
+ * hbl_launch_count: kernels this library has launched since it was loaded.
+ * hbl_profile_events: start_events / stop_events are HOST arrays of n cudaEvent_t
+ * handles owned by the caller; from now on the i-th launch of the selected kernel
+ * (1 = activation transform+quantize of Eq. 3-6, 2 = contraction+rescale of Eq. 7,
+ * 3 = weight unpack, 4 unused) is bracketed by cudaEventRecord(start[i]) /
+ * cudaEventRecord(stop[i]) on the launch's stream, until n pairs are used.
+ * kernel = 0 switches it off.  Returns the number of pairs the previous
+ * selection used (>= 0), or -status on an argument error. */
+unsigned long long hbl_launch_count(void);
+int hbl_profile_events(void** start_events, void** stop_events, int n, int kernel);
+
 /* Synchronises `stream`, returns the first device-side error recorded since the
  * last call (HBL_OK if none) and clears it. */
 int hbl_check_status(void* stream);

@@ -373,7 +373,10 @@ int launch_one(const void* x, int x_dtype, int T, int bits, float eps, int8_t* c
     }
   }
   const int grid = (T + TPC - 1) / TPC;
+  profile_before(KERNEL_ACT, s);
   kern<<<grid, THREADS, smem, s>>>(x, x_dtype == HBL_BF16, T, bits, eps, codes, scale, codesum, xr_out, zf, zw);
+  profile_after(KERNEL_ACT, s);
+  note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
 }
@@ -405,8 +408,11 @@ int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use
   }
   if (use_hadamard) return HBL_ERR_NOT_POW2;
   if (xr_out != nullptr) return HBL_ERR_SHAPE;
+  profile_before(KERNEL_ACT, s);
   act_quant_generic_kernel<<<T, 256, 0, s>>>(x, x_dtype == HBL_BF16, T, K, bits, eps, codes, scale, codesum,
                                              zero_fill, zero_fill_words);
+  profile_after(KERNEL_ACT, s);
+  note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
 }

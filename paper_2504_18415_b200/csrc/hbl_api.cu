@@ -11,9 +11,33 @@ namespace {
 __device__ int g_status = 0;
 }
 int* device_status_word() {
-  void* p = nullptr;
-  if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess) return nullptr;
-  return static_cast<int*>(p);
+  // One address per device; looked up once per device (a process may use several).
+  static int* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (cached[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess) return nullptr;
+    cached[dev] = static_cast<int*>(p);
+  }
+  return cached[dev];
+}
+
+namespace {
+unsigned long long g_launches = 0;
+struct Profile { void** starts = nullptr; void** stops = nullptr; int n = 0, next = 0, kernel = 0; bool open = false; } g_prof;
+}
+void note_launch() { ++g_launches; }
+void profile_before(int kernel_id, cudaStream_t s) {
+  if (g_prof.kernel != kernel_id || g_prof.next >= g_prof.n) return;
+  cudaEventRecord(static_cast<cudaEvent_t>(g_prof.starts[g_prof.next]), s);
+  g_prof.open = true;
+}
+void profile_after(int kernel_id, cudaStream_t s) {
+  if (g_prof.kernel != kernel_id || !g_prof.open) return;
+  cudaEventRecord(static_cast<cudaEvent_t>(g_prof.stops[g_prof.next]), s);
+  g_prof.open = false;
+  ++g_prof.next;
 }
 }  // namespace hbl
 
@@ -246,6 +270,35 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
                   reinterpret_cast<int*>(ws + w.counters[i]), reinterpret_cast<int8_t*>(ws + w.w_i8), s);
     if (rc != HBL_OK) return rc;
   }
+  return HBL_OK;
+}
+
+unsigned long long hbl_launch_count(void) { return g_launches; }
+
+int hbl_profile_events(void** start_events, void** stop_events, int n, int kernel) {
+  if (n < 0 || kernel < 0 || kernel > KERNEL_WEIGHT) return -HBL_ERR_SHAPE;
+  if (n > 0 && kernel != 0 && (!start_events || !stop_events)) return -HBL_ERR_NULL;
+  const int used = g_prof.next;
+  g_prof.starts = start_events; g_prof.stops = stop_events;
+  g_prof.n = (kernel == 0) ? 0 : n; g_prof.next = 0; g_prof.kernel = kernel; g_prof.open = false;
+  return used;
+}
+
+int hbl_forward_host(const void* x_host, int x_dtype, int tokens, int in_dim, const void* W_packed,
+                     const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y_host,
+                     void* x_stage, void* y_stage, void* workspace, size_t workspace_bytes, int path,
+                     void* stream) {
+  if (tokens < 0) return HBL_ERR_SHAPE;
+  if (tokens > 0 && (!x_host || !y_host || !x_stage || !y_stage)) return HBL_ERR_NULL;
+  if (x_dtype != HBL_F32 && x_dtype != HBL_BF16) return HBL_ERR_FORMAT;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t xb = (size_t)tokens * in_dim * (x_dtype == HBL_F32 ? 4 : 2);
+  const size_t yb = (size_t)tokens * out_dim * 2;
+  if (tokens > 0) HBL_CUDA_OK(cudaMemcpyAsync(x_stage, x_host, xb, cudaMemcpyHostToDevice, s));
+  int rc = hbl_forward(x_stage, x_dtype, tokens, in_dim, W_packed, alpha, out_dim, bits, use_hadamard, eps,
+                       y_stage, workspace, workspace_bytes, path, stream);
+  if (rc != HBL_OK) return rc;
+  if (tokens > 0) HBL_CUDA_OK(cudaMemcpyAsync(y_host, y_stage, yb, cudaMemcpyDeviceToHost, s));
   return HBL_OK;
 }
 

@@ -15,6 +15,12 @@ namespace hbl {
 int* device_status_word();
 __device__ __forceinline__ void report_device_error(int* status, int code) { atomicCAS(status, 0, code); }
 
+// ---- instrumentation (host side, see hbl_profile_events / hbl_launch_count) ----
+enum KernelId { KERNEL_NONE = 0, KERNEL_ACT = 1, KERNEL_CONTRACT = 2, KERNEL_UNPACK = 3, KERNEL_WEIGHT = 4 };
+void note_launch();                                   // +1 on the library's kernel-launch counter
+void profile_before(int kernel_id, cudaStream_t s);   // records the next start event if this kernel is selected
+void profile_after(int kernel_id, cudaStream_t s);
+
 // ---- small helpers ----------------------------------------------------------
 __host__ __device__ constexpr int ilog2(unsigned v) { return v <= 1 ? 0 : 1 + ilog2(v >> 1); }
 inline bool is_pow2(long v) { return v > 0 && (v & (v - 1)) == 0; }

@@ -203,9 +203,12 @@ int launch_nt(const int8_t* codes, const float* scale, const int32_t* codesum, i
   const int row_groups = (N + kRowsPerCta - 1) / kRowsPerCta;
   const size_t smem = (size_t)8 * NT * (Kc + 16);
   auto kern = gemm_stream_kernel<NT>;
+  profile_before(KERNEL_CONTRACT, s);
   kern<<<row_groups * splits, kWarps * 32, smem, s>>>(codes, scale, codesum, T, K, Kc,
                                                       static_cast<const uint4*>(Wp), N, alpha, y, acc_out,
                                                       acc_ws, counters);
+  profile_after(KERNEL_CONTRACT, s);
+  note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
 }

@@ -330,7 +330,10 @@ int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, co
   if (status == nullptr) return HBL_ERR_CUDA;
   const int n_tiles = ((T + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
+  profile_before(KERNEL_CONTRACT, s);
   gemm_tensor_kernel<<<grid, THREADS, SMEM_BYTES, s>>>(tmA, tmB, scale, alpha, y, acc_out, T, N, K, status);
+  profile_after(KERNEL_CONTRACT, s);
+  note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
 }

@@ -132,11 +132,13 @@ int launch_weight_quant(const void* W, int w_dtype, int N, int K, float eps, voi
   if (grid < 1) grid = 1;
   double* partials = static_cast<double*>(ws);
   absmean_partial_kernel<<<grid, kReduceThreads, 0, s>>>(W, w_dtype == HBL_BF16, total, partials);
+  note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   const size_t n_items = total / 16;
   int grid2 = (int)min((size_t)148 * 16, (n_items + 255) / 256);
   ternarise_pack_kernel<<<grid2, 256, 0, s>>>(W, w_dtype == HBL_BF16, N, K, eps, partials, grid,
                                               static_cast<uint4*>(packed), alpha);
+  note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
 }
@@ -144,7 +146,10 @@ int launch_weight_quant(const void* W, int w_dtype, int N, int K, float eps, voi
 int launch_unpack_weights(const void* packed, int N, int K, int8_t* out, cudaStream_t s) {
   const size_t n_items = (size_t)N * K / 16;
   int grid = (int)min((size_t)148 * 16, (n_items + 255) / 256);
+  profile_before(KERNEL_UNPACK, s);
   unpack_kernel<<<grid, 256, 0, s>>>(static_cast<const uint4*>(packed), N, K, out);
+  profile_after(KERNEL_UNPACK, s);
+  note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
 }

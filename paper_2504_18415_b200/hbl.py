@@ -26,7 +26,8 @@ EXPORTS = [
     "hbl_status_string", "hbl_packed_weight_bytes", "hbl_workspace_bytes",
     "hbl_quantize_weights_workspace_bytes", "hbl_quantize_weights", "hbl_forward",
     "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32",
-    "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights",
+    "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
+    "hbl_profile_events",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -72,6 +73,12 @@ def lib() -> C.CDLL:
         L.hbl_quantize_act.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp]
         L.hbl_gemm_i32.argtypes = [vp, vp, i, i, vp, i, vp, vp, sz, i, vp]
         L.hbl_unpack_weights.argtypes = [vp, i, i, vp, vp]
+        L.hbl_forward_host.argtypes = [vp, i, i, i, vp, vp, i, i, i, f, vp, vp, vp, vp, sz, i, vp]
+        L.hbl_forward_host.restype = C.c_int
+        L.hbl_launch_count.restype = C.c_ulonglong
+        L.hbl_launch_count.argtypes = []
+        L.hbl_profile_events.argtypes = [C.POINTER(vp), C.POINTER(vp), i, i]
+        L.hbl_profile_events.restype = C.c_int
         for n in ("hbl_quantize_weights", "hbl_forward", "hbl_block_forward", "hbl_check_status",
                   "hbl_hadamard_f32", "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights"):
             getattr(L, n).restype = C.c_int
@@ -216,3 +223,50 @@ def hbl_unpack_weights(W_packed: torch.Tensor, out_dim: int, in_dim: int) -> tor
     out = torch.empty((out_dim, in_dim), dtype=torch.int8, device=W_packed.device)
     _check(lib().hbl_unpack_weights(_ptr(W_packed), out_dim, in_dim, _ptr(out), _stream()), "hbl_unpack_weights")
     return out
+
+
+def hbl_forward_host(x_host: torch.Tensor, W_packed: torch.Tensor, alpha: torch.Tensor, out_dim: int,
+                     bits: int, use_hadamard: bool, y_host: torch.Tensor, x_stage: torch.Tensor,
+                     y_stage: torch.Tensor, workspace: torch.Tensor, eps: float = 1e-5,
+                     path: int = PATH_AUTO) -> torch.Tensor:
+    """hbl_forward with host-resident (pinned) x and y; copies are enqueued on the current stream."""
+    T, K = x_host.shape
+    if x_host.is_cuda or y_host.is_cuda:
+        raise ValueError("x_host / y_host must be host tensors")
+    _check(lib().hbl_forward_host(C.c_void_p(x_host.data_ptr()), _dt(x_host), T, K, _ptr(W_packed), _ptr(alpha),
+                                  out_dim, bits, int(bool(use_hadamard)), eps, C.c_void_p(y_host.data_ptr()),
+                                  _ptr(x_stage), _ptr(y_stage), _ptr(workspace), workspace.numel(), path,
+                                  _stream()), "hbl_forward_host")
+    return y_host
+
+
+def hbl_launch_count() -> int:
+    return int(lib().hbl_launch_count())
+
+
+class KernelTimer:
+    """Brackets the next n launches of one kernel class (1 = activation, 2 = contraction, 3 = unpack)
+    with CUDA events recorded by the library on the launching stream."""
+
+    def __init__(self, n: int, kernel: int):
+        self.n, self.kernel = n, kernel
+        self.starts = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        self.stops = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in self.starts + self.stops:      # torch creates the handle lazily, on first record
+            e.record()
+        self._a = (C.c_void_p * n)(*[e.cuda_event for e in self.starts])
+        self._b = (C.c_void_p * n)(*[e.cuda_event for e in self.stops])
+        self.used = 0
+
+    def __enter__(self):
+        rc = lib().hbl_profile_events(self._a, self._b, self.n, self.kernel)
+        if rc < 0:
+            raise HblError(-rc, "hbl_profile_events")
+        return self
+
+    def __exit__(self, *exc):
+        self.used = lib().hbl_profile_events(None, None, 0, 0)
+
+    def times_ms(self):
+        torch.cuda.synchronize()
+        return [self.starts[i].elapsed_time(self.stops[i]) for i in range(self.used)]
