@@ -335,6 +335,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", default="quick", choices=["none", "quick", "full"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default="", help="comma-separated point filters 'name-substring:tokens' "
+                    "(e.g. config4_a8_N32768:16,block:1); the sweep then runs just those points")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -459,7 +461,13 @@ def main():
         del xs, ys, work
         torch.cuda.empty_cache()
         full = args.sweep == "full"
-        L = lambda *a, **k: points.append(layer_point(*a, torch=torch, hbl=hbl, peaks=peaks, **k))
+        only = [f.split(":") for f in args.only.split(",") if f]
+        want = lambda name, T_: (not only) or any(o[0] in name and (len(o) < 2 or int(o[1]) == T_) for o in only)
+
+        def L(name, kind, seed, K_, N_, bits, had, T_):
+            if want(name, T_):
+                points.append(layer_point(name, kind, seed, K_, N_, bits, had, T_, torch=torch, hbl=hbl, peaks=peaks))
+
         for T_ in (1, 16, 256, 4096):
             L("config2_Wo_1p3B", "attn_out", 2, 2048, 2048, 4, True, T_)
         for T_ in (1, 16, 1024):
@@ -468,7 +476,8 @@ def main():
             for T_ in ((16, 4096, 32768) if full else (16, 4096)):
                 L(f"config4_a8_N{N_}", "gauss", 4, 4096, N_, 8, False, T_)
         for T_ in ((1, 4, 16, 64, 256, 1024, 4096, 16384, 65536) if full else (1, 16, 256, 4096)):
-            points.append(block_point(T_, torch, hbl, peaks))
+            if want("config5_block_7B", T_):
+                points.append(block_point(T_, torch, hbl, peaks))
 
     cpu = None
     if not args.no_cpu_baseline:

@@ -400,6 +400,8 @@ int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use
                      int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
                      int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s) {
   if (T <= 0) return HBL_OK;
+  if (use_hadamard && x_dtype == HBL_BF16 && act_quant_bf16_supported(K))
+    return launch_act_quant_bf16(x, T, K, bits, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s);
   if (is_pow2(K)) {
     const int m = ilog2((unsigned)K);
     return use_hadamard

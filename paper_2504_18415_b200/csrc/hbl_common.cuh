@@ -38,6 +38,11 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use_hadamard, float eps,
                      int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
                      int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s);
+// The same for bf16 inputs with the transform on (tensor-core first stages, packed fp32 butterflies).
+bool act_quant_bf16_supported(int K);
+int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
+                          int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
+                          cudaStream_t s);
 // Weight side: Eq. 1-2 and the 2-bit format.
 int launch_weight_quant(const void* W, int w_dtype, int N, int K, float eps, void* packed, float* alpha,
                         void* ws, cudaStream_t s);
