@@ -29,36 +29,62 @@ namespace {
 constexpr float kSqrt7 = 2.6457513110645906f;
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23: x + kMagic has rint(x) in its low mantissa bits
 
-// ---- packed fp32 pairs ---------------------------------------------------------
-__device__ __forceinline__ void butterfly2(float2& a, float2& b) {
-  float2 s, d;
-  asm("{\n .reg .b64 ra, rb, rs, rd;\n mov.b64 ra, {%4, %5};\n mov.b64 rb, {%6, %7};\n"
-      " add.rn.f32x2 rs, ra, rb;\n sub.rn.f32x2 rd, ra, rb;\n"
-      " mov.b64 {%0, %1}, rs;\n mov.b64 {%2, %3}, rd;\n}"
-      : "=f"(s.x), "=f"(s.y), "=f"(d.x), "=f"(d.y)
-      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+// ---- packed fp32 pairs, kept in 64-bit registers so that no pack/unpack moves are needed ----
+typedef unsigned long long f32x2_t;
+
+__device__ __forceinline__ f32x2_t pack2(float lo, float hi) {
+  f32x2_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// (a, b) -> (a + b, a - b) on both halves.  The difference is fma(b, -1, a): one packed
+// instruction with the same rounding as a subtraction.  `minus_one2` must live in a register
+// pair for the whole kernel (see opaque_minus_one2): as a literal it is re-created before every use.
+__device__ __forceinline__ void butterfly2(f32x2_t& a, f32x2_t& b, f32x2_t minus_one2) {
+  f32x2_t s, d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(s) : "l"(a), "l"(b));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(b), "l"(minus_one2), "l"(a));
   a = s;
   b = d;
+}
+__device__ __forceinline__ f32x2_t opaque_minus_one2() {
+  f32x2_t r;
+  asm volatile("mov.b64 %0, 0xBF800000BF800000;" : "=l"(r));
+  return r;
+}
+__device__ __forceinline__ f32x2_t fma2(f32x2_t a, f32x2_t b, f32x2_t c) {
+  f32x2_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {
+  float r;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
 }
 
 // Butterfly stages over bits [B0, B1) of the pair index (v holds 32 pairs).
 template <int B0, int B1>
-__device__ __forceinline__ void stages2(float2 (&v)[32]) {
+__device__ __forceinline__ void stages2(f32x2_t (&v)[32], f32x2_t minus_one2) {
 #pragma unroll
   for (int b = B0; b < B1; ++b) {
 #pragma unroll
     for (int e = 0; e < 32; ++e) {
       if ((e >> b) & 1) continue;
-      butterfly2(v[e], v[e | (1 << b)]);
+      butterfly2(v[e], v[e | (1 << b)], minus_one2);
     }
   }
 }
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{0f00000000, 0f00000000, 0f00000000, 0f00000000};"
       : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // Word address swizzle of a token's exchange buffer: toggles bit 2 with bits 5 and 8,
@@ -108,7 +134,7 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int group, in
 }
 
 template <int M, int BITS>
-__global__ void __launch_bounds__(Geometry<M>::THREADS, 512 / Geometry<M>::THREADS)
+__global__ void __launch_bounds__(Geometry<M>::THREADS, 768 / Geometry<M>::THREADS)
 fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
                        float* __restrict__ scale, int32_t* __restrict__ codesum, float* __restrict__ xr_out,
                        int32_t* __restrict__ zero_fill, size_t zero_words) {
@@ -127,8 +153,9 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   const int tid = tid_cta % NT;
   const int lane = tid_cta & 31, warp_cta = tid_cta >> 5;
   const int warp = tid >> 5;                               // warp inside the token group
-  const long token = (long)blockIdx.x * TPC + group;
-  const bool live = token < T;
+  const long token_raw = (long)blockIdx.x * TPC + group;
+  const bool live = token_raw < T;
+  const long token = live ? token_raw : (long)T - 1;       // a dead group recomputes the last token, stores nothing
   float* buf = smem + (size_t)group * K;
 
   // ---- the 16x16 sign matrix as B fragments (two MMAs: output columns 0-7 and 8-15) ----
@@ -151,13 +178,13 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
 
   // ---- phase 0: eight coalesced 16-byte chunks per lane; chunk c covers index
   //      c << (M-3) | warp << 8 | lane << 3 | m,  m = 0..7 ----
-  float2 v[32];
+  f32x2_t v[32];
   {
     const __nv_bfloat16* src = x + token * K + (warp << 8) + (lane << 3);
     uint4 raw[8];
 #pragma unroll
     for (int c = 0; c < 8; ++c)
-      raw[c] = live ? __ldg(reinterpret_cast<const uint4*>(src + ((size_t)c << (M - 3)))) : make_uint4(0, 0, 0, 0);
+      raw[c] = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)c << (M - 3))));
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
       // A fragment: (x: m 0,1) rows g, k3 = 0; (z: m 4,5) rows g+8; (y: m 2,3) k3 = 1; (w: m 6,7) both
@@ -166,22 +193,29 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
         float d[4];
         mma_bf16_16816(d, raw[c].x, raw[c].z, raw[c].y, raw[c].w, hb[j][0], hb[j][1]);
         // d[2h + b] is position m = b + 2j + 4h; pair index p = j + 2h
-        v[c * 4 + j] = make_float2(d[0], d[1]);
-        v[c * 4 + j + 2] = make_float2(d[2], d[3]);
+        v[c * 4 + j] = pack2(d[0], d[1]);
+        v[c * 4 + j + 2] = pack2(d[2], d[3]);
       }
     }
   }
   // pair index e = c*4 + p: bit 0 = index bit 1 (done), bit 1 = index bit 2, bits 2..4 = the chunk bits
-  stages2<1, 5>(v);
+  const f32x2_t minus_one2 = opaque_minus_one2();
+  stages2<1, 5>(v, minus_one2);
 
   // ---- exchange ----
+  // Swizzled addresses are (thread part) ^ (compile-time part); the two parts meet in bit 2
+  // only, so two base registers cover every case and the rest is an immediate offset.
+  const uint32_t sbuf = static_cast<uint32_t>(__cvta_generic_to_shared(buf));
   {
-    const int base = (warp << 8) | (lane << 3);
+    const uint32_t b0 = sbuf + 4u * swz_word((warp << 8) | (lane << 3));
+    const uint32_t b1 = b0 ^ 16u;                          // word bit 2 toggled
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-      const int a = swz_word(base | (c << (M - 3)));
-      *reinterpret_cast<float4*>(buf + a) = make_float4(v[c * 4].x, v[c * 4].y, v[c * 4 + 1].x, v[c * 4 + 1].y);
-      *reinterpret_cast<float4*>(buf + (a ^ 4)) = make_float4(v[c * 4 + 2].x, v[c * 4 + 2].y, v[c * 4 + 3].x, v[c * 4 + 3].y);
+      const int off = c << (M - 3);
+      const bool flip = ((off >> 5) ^ (off >> 8)) & 1;     // the chunk's own swizzle contribution
+      const uint32_t lo = (flip ? b1 : b0) + 4u * off, hi = (flip ? b0 : b1) + 4u * off;
+      asm volatile("st.shared.v2.b64 [%0], {%1, %2};" ::"r"(lo), "l"(v[c * 4]), "l"(v[c * 4 + 1]) : "memory");
+      asm volatile("st.shared.v2.b64 [%0], {%1, %2};" ::"r"(hi), "l"(v[c * 4 + 2]), "l"(v[c * 4 + 3]) : "memory");
     }
   }
   __syncthreads();
@@ -189,30 +223,62 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   // ---- final layout: local j (6 bits): low C bits = index bits [0,C), high R bits = index bits [5,5+R) ----
   const int fbase = ((tid & ((1 << (5 - C)) - 1)) << C) | ((tid >> (5 - C)) << (M - 3));
   auto findex = [&](int j) { return fbase | (j & (RUN - 1)) | ((j >> C) << 5); };
+  {
+    const uint32_t f0 = sbuf + 4u * swz_word(fbase);
+    const uint32_t f1 = f0 ^ 16u;
 #pragma unroll
-  for (int jh = 0; jh < (1 << R); ++jh) {
-    const int a = swz_word(fbase | (jh << 5));
-    if constexpr (C == 3) {
-      const float4 q0 = *reinterpret_cast<const float4*>(buf + a);
-      const float4 q1 = *reinterpret_cast<const float4*>(buf + (a ^ 4));
-      v[jh * 4 + 0] = make_float2(q0.x, q0.y); v[jh * 4 + 1] = make_float2(q0.z, q0.w);
-      v[jh * 4 + 2] = make_float2(q1.x, q1.y); v[jh * 4 + 3] = make_float2(q1.z, q1.w);
-    } else if constexpr (C == 2) {
-      const float4 q0 = *reinterpret_cast<const float4*>(buf + a);
-      v[jh * 2 + 0] = make_float2(q0.x, q0.y); v[jh * 2 + 1] = make_float2(q0.z, q0.w);
-    } else if constexpr (C == 1) {
-      v[jh] = *reinterpret_cast<const float2*>(buf + a);
-    } else {
-      if (jh & 1) v[jh >> 1].y = buf[a]; else v[jh >> 1].x = buf[a];
+    for (int jh = 0; jh < (1 << R); ++jh) {
+      const int off = jh << 5;
+      const bool flip = ((off >> 5) ^ (off >> 8)) & 1;
+      const uint32_t a = (flip ? f1 : f0) + 4u * off, a_hi = (flip ? f0 : f1) + 4u * off;
+      if constexpr (C == 3) {
+        asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(v[jh * 4]), "=l"(v[jh * 4 + 1]) : "r"(a));
+        asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(v[jh * 4 + 2]), "=l"(v[jh * 4 + 3]) : "r"(a_hi));
+      } else if constexpr (C == 2) {
+        asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(v[jh * 2]), "=l"(v[jh * 2 + 1]) : "r"(a));
+      } else if constexpr (C == 1) {
+        asm volatile("ld.shared.b64 %0, [%1];" : "=l"(v[jh]) : "r"(a));
+      } else {
+        if ((jh & 1) == 0) {                               // local bit 0 = index bit 5: elements jh, jh+1 form a pair
+          const int off1 = (jh + 1) << 5;
+          const bool flip1 = ((off1 >> 5) ^ (off1 >> 8)) & 1;
+          float lo, hi;
+          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(lo) : "r"(a));
+          asm volatile("ld.shared.f32 %0, [%1];" : "=f"(hi) : "r"((flip1 ? f1 : f0) + 4u * off1));
+          v[jh >> 1] = pack2(lo, hi);
+        }
+      }
     }
   }
+  // All stages but the last one (pair-index bit 4).
   if constexpr (C == 0) {
     // local bit 0 is index bit 5: that stage works inside each pair
 #pragma unroll
-    for (int e = 0; e < 32; ++e) v[e] = make_float2(v[e].x + v[e].y, v[e].x - v[e].y);
-    stages2<0, 5>(v);
+    for (int e = 0; e < 32; ++e) {
+      float lo, hi;
+      unpack2(v[e], lo, hi);
+      v[e] = pack2(lo + hi, lo - hi);
+    }
+    stages2<0, 4>(v, minus_one2);
   } else {
-    stages2<C - 1, 5>(v);      // pair-index bits [C-1, 5) are local bits [C, 6)
+    stages2<C - 1, 4>(v, minus_one2);      // pair-index bits [C-1, 5) are local bits [C, 6)
+  }
+  // Last stage, with the statistic's raw material taken from its inputs:
+  //   |a+b| + |a-b| = 2 max(|a|,|b|)   and   max(|a+b|,|a-b|) = |a| + |b|.
+  float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    float ax, ay, bx, by;
+    unpack2(v[e], ax, ay);
+    unpack2(v[e + 16], bx, by);
+    if constexpr (BITS == 8) {
+      s0 = fmaxf(s0, fabsf(ax) + fabsf(bx));
+      s1 = fmaxf(s1, fabsf(ay) + fabsf(by));
+    } else {
+      s0 += fmaxf(fabsf(ax), fabsf(bx));
+      s1 += fmaxf(fabsf(ay), fabsf(by));
+    }
+    butterfly2(v[e], v[e + 16], minus_one2);
   }
 
   constexpr float norm = G::NORM;
@@ -220,12 +286,14 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
     if (live) {
 #pragma unroll
       for (int e = 0; e < 32; ++e) {
+        float lo, hi;
+        unpack2(v[e], lo, hi);
         float* dst = xr_out + token * K + findex(2 * e);
         if constexpr (C >= 1) {
-          *reinterpret_cast<float2*>(dst) = make_float2(v[e].x * norm, v[e].y * norm);
+          *reinterpret_cast<float2*>(dst) = make_float2(lo * norm, hi * norm);
         } else {
-          dst[0] = v[e].x * norm;
-          xr_out[token * K + findex(2 * e + 1)] = v[e].y * norm;
+          dst[0] = lo * norm;
+          xr_out[token * K + findex(2 * e + 1)] = hi * norm;
         }
       }
     }
@@ -235,18 +303,10 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   // ---- per-token statistic (Eq. 5: max |x_r|; Eq. 6: mean |x_r|) ----
   float st;
   if constexpr (BITS == 8) {
-    float m0 = 0.f, m1 = 0.f;
-#pragma unroll
-    for (int e = 0; e < 32; ++e) { m0 = fmaxf(m0, fabsf(v[e].x)); m1 = fmaxf(m1, fabsf(v[e].y)); }
-    st = group_reduce<NT, true>(fmaxf(m0, m1), red_f, group, lane, warp_cta) * norm;
+    st = group_reduce<NT, true>(fmaxf(s0, s1), red_f, group, lane, warp_cta) * norm;
   } else {
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-    for (int e = 0; e < 32; e += 2) {
-      s0 += fabsf(v[e].x); s1 += fabsf(v[e].y); s2 += fabsf(v[e + 1].x); s3 += fabsf(v[e + 1].y);
-    }
-    const float s = group_reduce<NT, false>((s0 + s1) + (s2 + s3), red_f, group, lane, warp_cta);
-    st = (s * norm) * (1.0f / (float)K);
+    const float s = group_reduce<NT, false>(s0 + s1, red_f, group, lane, warp_cta);
+    st = ((2.0f * s) * norm) * (1.0f / (float)K);
   }
   constexpr float cq = (BITS == 8) ? 127.0f : kSqrt7;
   const float rq = __fdiv_rn(cq, st + eps) * norm;
@@ -254,40 +314,60 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   // ---- quantize; the low byte of (y + kMagic) is the code ----
   // (all reads of the exchange buffer happened before the barrier inside group_reduce)
   unsigned char* cbuf = reinterpret_cast<unsigned char*>(buf);
-  const float2 rq2 = make_float2(rq, rq), magic2 = make_float2(kMagic, kMagic);
-  uint32_t cb[32];               // per pair: code of .x in byte 0, code of .y in byte 1
+  uint32_t cb[32];               // per pair: code of the low element in byte 0, of the high one in byte 1
+  if constexpr (BITS == 8) {
+    const f32x2_t rq2 = pack2(rq, rq), magic2 = pack2(kMagic, kMagic);
 #pragma unroll
-  for (int e = 0; e < 32; ++e) {
-    float2 y;
-    if constexpr (BITS == 8) {
-      y = __ffma2_rn(v[e], rq2, magic2);      // |x_r| * rq < 127: no clip needed
-    } else {
-      y = __fmul2_rn(v[e], rq2);
-      y.x = fminf(fmaxf(y.x, -8.0f), 7.0f);
-      y.y = fminf(fmaxf(y.y, -8.0f), 7.0f);
-      y = __fadd2_rn(y, magic2);
+    for (int e = 0; e < 32; ++e) {
+      float lo, hi;
+      unpack2(fma2(v[e], rq2, magic2), lo, hi);   // |x_r| * rq < 127.5: no clip needed
+      cb[e] = __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x0040);
     }
-    cb[e] = __byte_perm(__float_as_uint(y.x), __float_as_uint(y.y), 0x0040);
+  } else {
+    // RoundClip(y, -8, 7) with y = x_r * rq: u = sat(y/15 + 8/15) is the clip (to [0,1]),
+    // 15 u - 8 + kMagic the rounding.  The two extra roundings move y by < 2e-6.
+    const float rq15 = rq * (1.0f / 15.0f);
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      float lo, hi;
+      unpack2(v[e], lo, hi);
+      lo = __fmaf_rn(fma_sat(lo, rq15, 8.0f / 15.0f), 15.0f, kMagic - 8.0f);
+      hi = __fmaf_rn(fma_sat(hi, rq15, 8.0f / 15.0f), 15.0f, kMagic - 8.0f);
+      cb[e] = __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x0040);
+    }
   }
+  // Staging byte address of element fbase | off(j): swz_code adds (index bits 9,10) << 5 onto bits 5,6,
+  // which always belong to off(j).  The thread's share of that is a 2-bit value tt, so four base
+  // registers (one per value of the offset's own bits 5,6) leave only immediates per store.
+  uint32_t cbase[4];
+  {
+    const uint32_t tt = (uint32_t)(fbase >> 9) & 3u;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) cbase[p] = sbuf + (uint32_t)fbase + (((uint32_t)p ^ tt) << 5);
+  }
+  auto caddr = [&](int j) {
+    const int off = (j & (RUN - 1)) | ((j >> C) << 5);
+    const int x = off ^ (((off >> 9) & 3) << 5);
+    return cbase[(x >> 5) & 3] + (uint32_t)(x & ~96);
+  };
   if constexpr (C == 0) {
 #pragma unroll
     for (int e = 0; e < 32; ++e) {
-      cbuf[swz_code(findex(2 * e))] = (unsigned char)(cb[e] & 0xFF);
-      cbuf[swz_code(findex(2 * e + 1))] = (unsigned char)(cb[e] >> 8);
+      asm volatile("st.shared.u8 [%0], %1;" ::"r"(caddr(2 * e)), "r"(cb[e]) : "memory");
+      asm volatile("st.shared.u8 [%0], %1;" ::"r"(caddr(2 * e + 1)), "r"(cb[e] >> 8) : "memory");
     }
   } else if constexpr (C == 1) {
 #pragma unroll
-    for (int e = 0; e < 32; ++e)
-      *reinterpret_cast<unsigned short*>(cbuf + swz_code(findex(2 * e))) = (unsigned short)cb[e];
+    for (int e = 0; e < 32; ++e) asm volatile("st.shared.u16 [%0], %1;" ::"r"(caddr(2 * e)), "h"((unsigned short)cb[e]) : "memory");
   } else if constexpr (C == 2) {
 #pragma unroll
     for (int e = 0; e < 32; e += 2)
-      *reinterpret_cast<uint32_t*>(cbuf + swz_code(findex(2 * e))) = __byte_perm(cb[e], cb[e + 1], 0x5410);
+      asm volatile("st.shared.u32 [%0], %1;" ::"r"(caddr(2 * e)), "r"(__byte_perm(cb[e], cb[e + 1], 0x5410)) : "memory");
   } else {
 #pragma unroll
     for (int e = 0; e < 32; e += 4)
-      *reinterpret_cast<uint2*>(cbuf + swz_code(findex(2 * e))) =
-          make_uint2(__byte_perm(cb[e], cb[e + 1], 0x5410), __byte_perm(cb[e + 2], cb[e + 3], 0x5410));
+      asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(caddr(2 * e)), "r"(__byte_perm(cb[e], cb[e + 1], 0x5410)),
+                   "r"(__byte_perm(cb[e + 2], cb[e + 3], 0x5410)) : "memory");
   }
   __syncthreads();
 
@@ -298,10 +378,12 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
     const int q = tid + r * NT;
     const uint4 w = *reinterpret_cast<const uint4*>(cbuf + swz_code(q << 4));
     if (live) *reinterpret_cast<uint4*>(codes + token * K + ((size_t)q << 4)) = w;
-    csum = __dp4a((int)w.x, 0x01010101, csum);
-    csum = __dp4a((int)w.y, 0x01010101, csum);
-    csum = __dp4a((int)w.z, 0x01010101, csum);
-    csum = __dp4a((int)w.w, 0x01010101, csum);
+    if (codesum != nullptr) {
+      csum = __dp4a((int)w.x, 0x01010101, csum);
+      csum = __dp4a((int)w.y, 0x01010101, csum);
+      csum = __dp4a((int)w.z, 0x01010101, csum);
+      csum = __dp4a((int)w.w, 0x01010101, csum);
+    }
   }
   if (codesum != nullptr) {      // uniform over the grid
 #pragma unroll

@@ -177,7 +177,8 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
   int32_t* codesum = reinterpret_cast<int32_t*>(ws + w.codesum);
   int8_t* codes = reinterpret_cast<int8_t*>(ws + w.codes);
   const bool stream_path = (p == HBL_PATH_STREAM);
-  rc = launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale, codesum, nullptr,
+  rc = launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale,
+                        stream_path ? codesum : nullptr /* only the streaming kernel needs the code sums */, nullptr,
                         stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
                         stream_path ? w.zero_words : 0, s);
   if (rc != HBL_OK) return rc;
@@ -255,7 +256,7 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   for (int i = 0; i < 4; ++i) {
     rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
                           reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
-                          reinterpret_cast<int32_t*>(ws + w.codesum[i]), nullptr,
+                          stream_path ? reinterpret_cast<int32_t*>(ws + w.codesum[i]) : nullptr, nullptr,
                           (stream_path && i == 0) ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
                           (stream_path && i == 0) ? w.zero_words : 0, s);
     if (rc != HBL_OK) return rc;
