@@ -159,6 +159,29 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
                  const void* W_packed, int out_dim, int32_t* acc_out,
                  void* workspace, size_t workspace_bytes, int path, void* stream);
 
+/* hbl_gemm_i32 on the streaming kernel for callers that cannot hand over a
+ * workspace.  (No counterpart in the paper: this is a packaging variant of the
+ * contraction above.)  Some hosts of this library may not allocate device memory
+ * at the point where they call it -- an inference server that gave every spare
+ * byte to its KV-cache pool at start-up, a plugin running inside a framework's
+ * stream callback where an allocation would synchronise the device, a runtime
+ * whose memory budget is frozen after initialisation -- and have no buffer of
+ * their own to lend.  For them the kernel's scratch (split-K partial sums and
+ * arrival counters) sits in a fixed 1 MiB + 4 KiB array inside the library's
+ * device image; every GPU that loads the library holds it until the process ends.
+ *   - Inputs and the output are still the caller's: codes int8 [T,K], codesum
+ *     int32 [T], W_packed, acc_out int32 [T,N], all device pointers.
+ *   - Limits: tokens <= 64, tokens * out_dim <= 262144, out_dim <= 131072; anything
+ *     larger returns HBL_ERR_TOO_LARGE before any work is enqueued.
+ *   - The call allocates and frees nothing.  The first call on each device looks up
+ *     the array's device address (that device must be current); make that first
+ *     call outside any stream capture.
+ *   - Every call reuses the same array and clears the part it needs on `stream`
+ *     first.  Two calls that can overlap on the GPU (different streams, no ordering
+ *     between them) race on it: order them. */
+int hbl_gemm_i32_static(const int8_t* codes, const int32_t* codesum, int tokens, int in_dim,
+                        const void* W_packed, int out_dim, int32_t* acc_out, void* stream);
+
 /* Packed ternary -> int8 [N,K] row-major, values in {-1,0,1}. */
 int hbl_unpack_weights(const void* W_packed, int out_dim, int in_dim, int8_t* w_out, void* stream);
 

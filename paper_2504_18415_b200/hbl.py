@@ -27,7 +27,7 @@ EXPORTS = [
     "hbl_quantize_weights_workspace_bytes", "hbl_quantize_weights", "hbl_forward",
     "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32",
     "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
-    "hbl_profile_events",
+    "hbl_profile_events", "hbl_gemm_i32_static",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -73,6 +73,8 @@ def lib() -> C.CDLL:
         L.hbl_quantize_act.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp]
         L.hbl_gemm_i32.argtypes = [vp, vp, i, i, vp, i, vp, vp, sz, i, vp]
         L.hbl_unpack_weights.argtypes = [vp, i, i, vp, vp]
+        L.hbl_gemm_i32_static.argtypes = [vp, vp, i, i, vp, i, vp, vp]
+        L.hbl_gemm_i32_static.restype = C.c_int
         L.hbl_forward_host.argtypes = [vp, i, i, i, vp, vp, i, i, i, f, vp, vp, vp, vp, sz, i, vp]
         L.hbl_forward_host.restype = C.c_int
         L.hbl_launch_count.restype = C.c_ulonglong
@@ -216,6 +218,17 @@ def hbl_gemm_i32(codes: torch.Tensor, codesum: torch.Tensor | None, W_packed: to
         workspace = new_workspace(hbl_workspace_bytes(T, K, out_dim), codes.device)
     _check(lib().hbl_gemm_i32(_ptr(codes), _ptr(codesum), T, K, _ptr(W_packed), out_dim, _ptr(acc),
                               _ptr(workspace), workspace.numel(), path, _stream()), "hbl_gemm_i32")
+    return acc
+
+
+def hbl_gemm_i32_static(codes: torch.Tensor, codesum: torch.Tensor, W_packed: torch.Tensor, out_dim: int) -> torch.Tensor:
+    """hbl_gemm_i32 (streaming kernel) without a workspace argument: for hosts that cannot allocate
+    or lend scratch memory, the scratch is a fixed array inside the library (see include/hbl.h for
+    the size limits).  Only the result tensor is created here, by torch, as for every other call."""
+    T, K = codes.shape
+    acc = torch.empty((T, out_dim), dtype=torch.int32, device=codes.device)
+    _check(lib().hbl_gemm_i32_static(_ptr(codes), _ptr(codesum), T, K, _ptr(W_packed), out_dim, _ptr(acc),
+                                     _stream()), "hbl_gemm_i32_static")
     return acc
 
 
