@@ -39,6 +39,8 @@ EPS = 1e-5
 L2_BYTES = 126 * 1024 * 1024
 RING_BYTES = 4 * L2_BYTES            # ring of distinct input sets so that every call is L2-cold
 NOMINAL_INT8_TOPS = 4500.0
+ALU_PEAK_LANE_OPS = 148 * 128 * 1.965e9      # fp32 lanes x SMs x clocks.max.sm
+GEMM_TENSOR_TRAFFIC_BYTES = 195293440        # 151.1 MB read + 44.2 MB written per launch (headline workload)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -129,6 +131,22 @@ def device_weights(N, K, seed, torch, hbl):
     packed, alpha = hbl.hbl_quantize_weights(W, EPS)
     del W
     return packed, alpha
+
+
+def max_over_ranks(total_ms, dist, device):
+    """Device time of the slowest rank (MAX all-reduce) followed by a barrier; identity without a group."""
+    if dist is None:
+        return float(total_ms)
+    import torch
+    t = torch.tensor([float(total_ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.barrier()
+    return float(t.item())
+
+
+def whole_job_value(world, tokens_per_rank, ms_per_step):
+    """tokens/s summed over `world` independent replicas that all ran the same step in ms_per_step."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
 def time_loop(fn, iters, warmup, torch):
@@ -391,11 +409,7 @@ def main():
         torch.cuda.synchronize()
     launches = hbl.hbl_launch_count() - launches0
     total_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.barrier()
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     torch.cuda.synchronize()
     # keep the GPU busy a little longer so that the clock sampler sees load
     if rank == 0:
@@ -410,7 +424,7 @@ def main():
     if st != 0:
         raise RuntimeError(f"device status {st}")
     ms_per_step = total_ms / Ksteps
-    value = world * T / (ms_per_step * 1e-3)
+    value = whole_job_value(world, T, ms_per_step)
 
     # per-kernel breakdown (outside the timed region)
     breakdown = {}
@@ -449,12 +463,21 @@ def main():
                 "traffic": None,
                 "note": f"int8 multiply-add = 2 ops; peak = 2 x {peak_src} bf16 burst (nominal int8:bf16 ratio); "
                         f"of nominal 4500: {ach / NOMINAL_INT8_TOPS:.3f}; kernel avg {gemm_ms * 1e3:.1f} us over {len(kt.times_ms())} launches"}
-    tr = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tr):
-        try:
-            roofline["traffic"] = json.load(open(tr)).get("gemm_tensor_kernel_bytes_per_launch")
-        except Exception:
-            pass
+    # DRAM bytes of one launch of this kernel at this workload, from the ncu capture summarised in
+    # profiles/gemm_tensor_kernel_config3_T16384.md (dram__bytes_read.sum + dram__bytes_write.sum).
+    # Set to None whenever the kernel changes until the counters are taken again.
+    roofline["traffic"] = GEMM_TENSOR_TRAFFIC_BYTES
+    act_ms = breakdown["act_quant_kernel"]
+    kernels = {
+        "fwht_quant_bf16_kernel": {
+            "ms": act_ms, "hbm_gbs": round(3.0 * T * K / (act_ms * 1e-3) / 1e9, 1),
+            "hbm_frac": round(3.0 * T * K / (act_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+            "alu_frac": round(12.5 * T * K / (act_ms * 1e-3) / ALU_PEAK_LANE_OPS, 4),
+            "note": "3 B of kernel traffic and 12.5 fp32 lane-ops per element; ALU peak 148 SMs x 128 lanes x 1.965 GHz"},
+        "unpack_kernel": {"ms": breakdown["unpack_kernel"],
+                          "hbm_frac": round(1.25 * N * K / (breakdown["unpack_kernel"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)},
+        "gemm_tensor_kernel": {"ms": breakdown["gemm_tensor_kernel"]},
+    }
 
     points = []
     if args.sweep != "none" and world == 1:
@@ -495,7 +518,7 @@ def main():
                    "parallelism": "replicas" if world > 1 else "single GPU"},
         "tops": round(ops / (ms_per_step * 1e-3) / 1e12, 2),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "kernels_ms": breakdown, "roofline": roofline, "cpu_baseline": cpu, "points": points,
+        "kernels_ms": breakdown, "kernels": kernels, "roofline": roofline, "cpu_baseline": cpu, "points": points,
         "peaks": {**peaks, "source": peak_src, "int8_nominal_tops": NOMINAL_INT8_TOPS},
     }
     print(json.dumps(out))
