@@ -177,10 +177,10 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
   int32_t* codesum = reinterpret_cast<int32_t*>(ws + w.codesum);
   int8_t* codes = reinterpret_cast<int8_t*>(ws + w.codes);
   const bool stream_path = (p == HBL_PATH_STREAM);
+  const bool zero = stream_path && gemm_stream_uses_scratch(tokens, in_dim, out_dim);
   rc = launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale,
                         stream_path ? codesum : nullptr /* only the streaming kernel needs the code sums */, nullptr,
-                        stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
-                        stream_path ? w.zero_words : 0, s);
+                        zero ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr, zero ? w.zero_words : 0, s);
   if (rc != HBL_OK) return rc;
   return run_gemm(p, codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha, y, nullptr,
                   reinterpret_cast<int32_t*>(ws + w.acc), reinterpret_cast<int*>(ws + w.counters),
@@ -253,16 +253,18 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   const int in_dims[4] = {H, H, H, F};
   const int had[4] = {0, 1, 0, 1};
   const bool stream_path = (p == HBL_PATH_STREAM);
+  const int src[7] = {0, 0, 0, 1, 2, 2, 3};                  // which quantized input feeds each projection
+  const int out_dims[7] = {H, H, H, H, F, F, H};
+  bool zero = false;                                         // does any projection combine partial sums in scratch?
+  for (int i = 0; i < 7 && stream_path; ++i) zero = zero || gemm_stream_uses_scratch(T, in_dims[src[i]], out_dims[i]);
   for (int i = 0; i < 4; ++i) {
     rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
                           reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
                           stream_path ? reinterpret_cast<int32_t*>(ws + w.codesum[i]) : nullptr, nullptr,
-                          (stream_path && i == 0) ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
-                          (stream_path && i == 0) ? w.zero_words : 0, s);
+                          (zero && i == 0) ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
+                          (zero && i == 0) ? w.zero_words : 0, s);
     if (rc != HBL_OK) return rc;
   }
-  const int src[7] = {0, 0, 0, 1, 2, 2, 3};                  // which quantized input feeds each projection
-  const int out_dims[7] = {H, H, H, H, F, F, H};
   for (int i = 0; i < 7; ++i) {
     const int xi = src[i];
     rc = run_gemm(p, reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]),

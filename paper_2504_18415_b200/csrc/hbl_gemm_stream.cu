@@ -216,7 +216,16 @@ int launch_nt(const int8_t* codes, const float* scale, const int32_t* codesum, i
 }  // namespace
 
 size_t gemm_stream_acc_words(int T, int N) { return (size_t)T * N; }
-size_t gemm_stream_counter_words(int N) { return (size_t)(N + kRowsPerCta - 1) / kRowsPerCta; }
+size_t gemm_stream_counter_words(int N) { return (size_t)(N + 15) / 16; }   // one per 16-row tile (covers both kernels)
+
+// True when the streaming contraction will combine partial sums in acc_ws / counters (which must
+// then be zero on entry); false when every output is finished inside one CTA.
+bool gemm_stream_uses_scratch(int T, int K, int N) {
+  if (T <= 0) return false;
+  if (gemm_kslice_supported(T, K)) return gemm_kslice_passes(T, K, N) > 1;
+  const int max_kc = T <= 16 ? 2048 : (T <= 32 ? 1024 : 512);
+  return K / choose_kc(N, K, max_kc) > 1;
+}
 
 // acc_ws [T*N] and counters must be zero on entry when K is split (the caller
 // clears them; the activation kernel does it as a side job in hbl_forward).
@@ -225,6 +234,8 @@ int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* c
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s) {
   if (T <= 0) return HBL_OK;
   if (T > 64) return HBL_ERR_TOO_LARGE;
+  if (gemm_kslice_supported(T, K))
+    return launch_gemm_kslice(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
   if (T <= 8) return launch_nt<1>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
   if (T <= 16) return launch_nt<2>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
   if (T <= 32) return launch_nt<4>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
