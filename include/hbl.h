@@ -167,11 +167,11 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
  * stream callback where an allocation would synchronise the device, a runtime
  * whose memory budget is frozen after initialisation -- and have no buffer of
  * their own to lend.  For them the kernel's scratch (split-K partial sums and
- * arrival counters) sits in a fixed 1 MiB + 32 KiB array inside the library's
+ * arrival counters) sits in a fixed 1 MiB + 4 KiB array inside the library's
  * device image; every GPU that loads the library holds it until the process ends.
  *   - Inputs and the output are still the caller's: codes int8 [T,K], codesum
  *     int32 [T], W_packed, acc_out int32 [T,N], all device pointers.
- *   - Limits: tokens <= 64, tokens (rounded up to 8, 16, 32 or 64) * out_dim <= 262144, out_dim <= 131072; anything
+ *   - Limits: tokens <= 64, tokens * out_dim <= 262144, out_dim <= 131072; anything
  *     larger returns HBL_ERR_TOO_LARGE before any work is enqueued.
  *   - The call allocates and frees nothing.  The first call on each device looks up
  *     the array's device address (that device must be current); make that first

@@ -177,11 +177,10 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
   int32_t* codesum = reinterpret_cast<int32_t*>(ws + w.codesum);
   int8_t* codes = reinterpret_cast<int8_t*>(ws + w.codes);
   const bool stream_path = (p == HBL_PATH_STREAM);
-  size_t zero = stream_path ? gemm_stream_zero_words(tokens, in_dim, out_dim) : 0;
-  if (zero > w.zero_words) zero = w.zero_words;
   rc = launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale,
                         stream_path ? codesum : nullptr /* only the streaming kernel needs the code sums */, nullptr,
-                        zero ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr, zero, s);
+                        stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
+                        stream_path ? w.zero_words : 0, s);
   if (rc != HBL_OK) return rc;
   return run_gemm(p, codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha, y, nullptr,
                   reinterpret_cast<int32_t*>(ws + w.acc), reinterpret_cast<int*>(ws + w.counters),
@@ -191,7 +190,7 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
 // ---- decoder block: four quantizations, seven projections -------------------------------
 namespace {
 struct BlockWs {
-  size_t scale[4], codesum[4], codes[4], zero_region, counters[7], acc[7], w_i8, total, zero_words, counter_words;
+  size_t scale[4], codesum[4], codes[4], zero_region, counters[7], acc[7], w_i8, total, zero_words;
 };
 BlockWs carve_block(int T, int H, int F) {
   BlockWs w{};
@@ -201,10 +200,11 @@ BlockWs carve_block(int T, int H, int F) {
   for (int i = 0; i < 4; ++i) { w.scale[i] = off; off = align_up(off + 4 * (size_t)T, 256); }
   for (int i = 0; i < 4; ++i) { w.codesum[i] = off; off = align_up(off + 4 * (size_t)T, 256); }
   const int ts = T < kStreamMaxTokens ? T : kStreamMaxTokens;
-  w.zero_region = off;                                       // all counters first: often only they need clearing
-  for (int i = 0; i < 7; ++i) { w.counters[i] = off; off += sizeof(int) * align_up(gemm_stream_counter_words(out_dims[i]), 4); }
-  w.counter_words = (off - w.zero_region) / 4;
-  for (int i = 0; i < 7; ++i) { w.acc[i] = off; off += sizeof(int32_t) * gemm_stream_acc_words(ts, out_dims[i]); }
+  w.zero_region = off;
+  for (int i = 0; i < 7; ++i) {
+    w.counters[i] = off; off += sizeof(int) * align_up(gemm_stream_counter_words(out_dims[i]), 4);
+    w.acc[i] = off;      off += sizeof(int32_t) * gemm_stream_acc_words(ts, out_dims[i]);
+  }
   w.zero_words = (off - w.zero_region) / 4;
   off = align_up(off, 1024);
   for (int i = 0; i < 4; ++i) { w.codes[i] = off; off = align_up(off + (size_t)T * in_dims[i], 1024); }
@@ -253,22 +253,16 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   const int in_dims[4] = {H, H, H, F};
   const int had[4] = {0, 1, 0, 1};
   const bool stream_path = (p == HBL_PATH_STREAM);
-  const int src[7] = {0, 0, 0, 1, 2, 2, 3};                  // which quantized input feeds each projection
-  const int out_dims[7] = {H, H, H, H, F, F, H};
-  size_t zero = 0;                                           // words of the scratch region the contractions need cleared
-  for (int i = 0; i < 7 && stream_path; ++i) {
-    const size_t z = gemm_stream_zero_words(T, in_dims[src[i]], out_dims[i]);
-    const size_t need = z == 0 ? 0 : (z <= gemm_stream_counter_words(out_dims[i]) ? w.counter_words : w.zero_words);
-    if (need > zero) zero = need;
-  }
   for (int i = 0; i < 4; ++i) {
     rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
                           reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
                           stream_path ? reinterpret_cast<int32_t*>(ws + w.codesum[i]) : nullptr, nullptr,
-                          (zero && i == 0) ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
-                          i == 0 ? zero : 0, s);
+                          (stream_path && i == 0) ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
+                          (stream_path && i == 0) ? w.zero_words : 0, s);
     if (rc != HBL_OK) return rc;
   }
+  const int src[7] = {0, 0, 0, 1, 2, 2, 3};                  // which quantized input feeds each projection
+  const int out_dims[7] = {H, H, H, H, F, F, H};
   for (int i = 0; i < 7; ++i) {
     const int xi = src[i];
     rc = run_gemm(p, reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]),

@@ -57,15 +57,9 @@ struct GemmSegment {          // one weight tensor of a (possibly fused) project
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
                        const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s);
-bool gemm_kslice_supported(int T, int K, int N);    // K-sliced persistent streaming kernel (T <= 32, K % 1024 == 0)
-int gemm_kslice_flag_words(int T, int K, int N);
-int launch_gemm_kslice(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
-                       const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
-                       int32_t* acc_out, int32_t* part, int* flags, cudaStream_t s);
 int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
                        const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s);
 size_t gemm_stream_acc_words(int T, int N);       // int32 words of split-K scratch (0 if none)
 size_t gemm_stream_counter_words(int N);
-size_t gemm_stream_zero_words(int T, int K, int N);   // words of the [counters][acc_ws] region that must be zero (SIZE_MAX = all)
 
 }  // namespace hbl

@@ -215,21 +215,8 @@ int launch_nt(const int8_t* codes, const float* scale, const int32_t* codesum, i
 
 }  // namespace
 
-// Tokens rounded up to the MMA padding (8, 16, 32, 64): covers T*N partial sums and the K-sliced kernel's part slots.
-size_t gemm_stream_acc_words(int T, int N) {
-  const int tp = T <= 8 ? 8 : (T <= 16 ? 16 : (T <= 32 ? 32 : 64));
-  return (size_t)tp * N;
-}
-size_t gemm_stream_counter_words(int N) { return (size_t)(N + 15) / 16; }   // one per 16-row tile (covers both kernels)
-
-// How many 32-bit words, counted from the start of the [counters][acc_ws] scratch region, must be
-// zero when the streaming contraction starts: 0 (none), a few flag words, or everything (SIZE_MAX).
-size_t gemm_stream_zero_words(int T, int K, int N) {
-  if (T <= 0) return 0;
-  if (gemm_kslice_supported(T, K, N)) return (size_t)gemm_kslice_flag_words(T, K, N);
-  const int max_kc = T <= 16 ? 2048 : (T <= 32 ? 1024 : 512);
-  return K / choose_kc(N, K, max_kc) > 1 ? (size_t)-1 : 0;
-}
+size_t gemm_stream_acc_words(int T, int N) { return (size_t)T * N; }
+size_t gemm_stream_counter_words(int N) { return (size_t)(N + kRowsPerCta - 1) / kRowsPerCta; }
 
 // acc_ws [T*N] and counters must be zero on entry when K is split (the caller
 // clears them; the activation kernel does it as a side job in hbl_forward).
@@ -238,8 +225,6 @@ int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* c
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s) {
   if (T <= 0) return HBL_OK;
   if (T > 64) return HBL_ERR_TOO_LARGE;
-  if (gemm_kslice_supported(T, K, N))
-    return launch_gemm_kslice(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
   if (T <= 8) return launch_nt<1>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
   if (T <= 16) return launch_nt<2>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
   if (T <= 32) return launch_nt<4>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);

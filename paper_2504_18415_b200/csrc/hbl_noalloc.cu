@@ -9,7 +9,7 @@ using namespace hbl;
 namespace {
 
 constexpr size_t kStaticAccWords = 262144;      // tokens * out_dim may not exceed this (1 MiB of int32)
-constexpr size_t kStaticCounterWords = 8192;    // one per 16-row tile: out_dim <= 131072
+constexpr size_t kStaticCounterWords = 1024;    // row groups of 128 outputs: out_dim <= 131072
 constexpr size_t kStaticScratchBytes = (kStaticAccWords + kStaticCounterWords) * sizeof(int32_t);
 
 // Every GPU that loads the library holds this array until the process exits.
