@@ -62,11 +62,12 @@ typedef enum {
 const char* hbl_status_string(int status);
 
 /* Bytes of the packed ternary weight tensor for W[out_dim, in_dim]: 2 bits per
- * weight, stored as u = w + 1 in {0,1,2}.  Layout: tiles of 16 rows x 128
- * columns, 512 bytes each, ordered [row tile][column tile]; inside a tile, 32
- * groups of four 32-bit words; word j of group l holds the 16 weights with
- * rows 16*tile + (l>>2) + 8*(i&1), columns 128*ctile + 32*j + 16*(i>>1) + 4*(l&3) + b
- * (i = 0..3, b = 0..3) at bit position 8*b + 2*i.  Returns 0 on bad shapes. */
+ * weight, stored as u = w + 1 in {0,1,2}, rows padded with zeros to a multiple of
+ * 128: ceil(out_dim/128)*128*in_dim/4 bytes.  Layout: tiles of 128 rows x 128
+ * columns, 4096 bytes each, ordered [row block][column block]; a tile is
+ * [h = 0,1][row 0..127][four 32-bit words]; word v of (h, row) holds the weights
+ * of row 128*rb + row in columns 128*kb + 16*(4h+v) + 4*i + b (i, b = 0..3) at
+ * bit position 8*b + 2*i.  Returns 0 on bad shapes. */
 size_t hbl_packed_weight_bytes(int out_dim, int in_dim);
 
 /* Scratch bytes hbl_forward needs for up to max_tokens tokens (any bits, any path). */
@@ -166,13 +167,14 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
  * byte to its KV-cache pool at start-up, a plugin running inside a framework's
  * stream callback where an allocation would synchronise the device, a runtime
  * whose memory budget is frozen after initialisation -- and have no buffer of
- * their own to lend.  For them the kernel's scratch (split-K partial sums and
- * arrival counters) sits in a fixed 1 MiB + 4 KiB array inside the library's
- * device image; every GPU that loads the library holds it until the process ends.
+ * their own to lend.  For them the kernel's scratch (partial sums handed between
+ * thread blocks, and their ready flags) sits in a fixed 1.25 MiB + 1 KiB array inside
+ * the library's device image; every GPU that loads the library holds it until the
+ * process ends.
  *   - Inputs and the output are still the caller's: codes int8 [T,K], codesum
  *     int32 [T], W_packed, acc_out int32 [T,N], all device pointers.
- *   - Limits: tokens <= 64, tokens * out_dim <= 262144, out_dim <= 131072; anything
- *     larger returns HBL_ERR_TOO_LARGE before any work is enqueued.
+ *   - Limit: tokens <= 16 (any out_dim); more tokens return HBL_ERR_TOO_LARGE before
+ *     any work is enqueued.
  *   - The call allocates and frees nothing.  The first call on each device looks up
  *     the array's device address (that device must be current); make that first
  *     call outside any stream capture.

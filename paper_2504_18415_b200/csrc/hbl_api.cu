@@ -57,10 +57,10 @@ ForwardWs carve(int T, int K, int N) {
   w.scale = off;   off = align_up(off + sizeof(float) * (size_t)T, 256);
   w.codesum = off; off = align_up(off + sizeof(int32_t) * (size_t)T, 256);
   const int ts = T < kStreamMaxTokens ? T : kStreamMaxTokens;
-  w.zero_region = off;
+  w.zero_region = off;                                      // only the flags must be zero when the contraction starts
   w.counters = off; off += sizeof(int) * align_up(gemm_stream_counter_words(N), 4);
-  w.acc = off;      off += sizeof(int32_t) * gemm_stream_acc_words(ts, N);
   w.zero_words = (off - w.zero_region) / 4;
+  w.acc = off;      off += sizeof(int32_t) * gemm_stream_acc_words(ts, N);
   off = align_up(off, 1024);
   w.codes = off;   off = align_up(off + (size_t)T * K, 1024);
   w.w_i8 = off;    off = align_up(off + (size_t)N * K, 1024);
@@ -126,7 +126,7 @@ const char* hbl_status_string(int status) {
 
 size_t hbl_packed_weight_bytes(int out_dim, int in_dim) {
   if (check_dims(0, in_dim, out_dim) != HBL_OK) return 0;
-  return (size_t)out_dim * in_dim / 4;
+  return (size_t)((out_dim + 127) / 128) * 128 * in_dim / 4;   // rows padded to whole 128-row tiles
 }
 
 size_t hbl_workspace_bytes(int max_tokens, int in_dim, int out_dim) {
@@ -200,12 +200,10 @@ BlockWs carve_block(int T, int H, int F) {
   for (int i = 0; i < 4; ++i) { w.scale[i] = off; off = align_up(off + 4 * (size_t)T, 256); }
   for (int i = 0; i < 4; ++i) { w.codesum[i] = off; off = align_up(off + 4 * (size_t)T, 256); }
   const int ts = T < kStreamMaxTokens ? T : kStreamMaxTokens;
-  w.zero_region = off;
-  for (int i = 0; i < 7; ++i) {
-    w.counters[i] = off; off += sizeof(int) * align_up(gemm_stream_counter_words(out_dims[i]), 4);
-    w.acc[i] = off;      off += sizeof(int32_t) * gemm_stream_acc_words(ts, out_dims[i]);
-  }
+  w.zero_region = off;                                      // the seven flag arrays first: only they must be zero
+  for (int i = 0; i < 7; ++i) { w.counters[i] = off; off += sizeof(int) * align_up(gemm_stream_counter_words(out_dims[i]), 4); }
   w.zero_words = (off - w.zero_region) / 4;
+  for (int i = 0; i < 7; ++i) { w.acc[i] = off; off += sizeof(int32_t) * gemm_stream_acc_words(ts, out_dims[i]); }
   off = align_up(off, 1024);
   for (int i = 0; i < 4; ++i) { w.codes[i] = off; off = align_up(off + (size_t)T * in_dims[i], 1024); }
   w.w_i8 = off; off = align_up(off + (size_t)F * H, 1024);   // largest weight: F x H

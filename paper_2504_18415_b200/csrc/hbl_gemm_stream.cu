@@ -1,212 +1,384 @@
-// Small-batch contraction of H-BitLinear (Eq. 7), weight-streaming bound.
+// Small-batch contraction of H-BitLinear (Eq. 7) for T <= 64 tokens, bound by the
+// stream of 2-bit packed weights out of HBM.
 //
-// At T <= 64 tokens every packed weight byte is used once and the call is bound
-// by how fast the 2-bit weights stream out of HBM.  Each warp reads its weight
-// tiles with 128-bit loads straight into registers (the packed format is the
-// register fragment order of the m16n8k32 integer MMA, see hbl_weights.cu),
-// widens 16 weights with four shift-and-mask operations and contracts them with
-// the tokens' int8 codes, which the CTA stages once in shared memory.  Nothing
-// but the packed bytes crosses shared memory or HBM on the weight side.
+// The roles are swapped with respect to the large-batch kernel: 128 weight rows
+// are the M side of tcgen05.mma kind::i8 and the (padded) tokens the N side, so a
+// step of 128 x T x 32 costs a few cycles of the tensor core and the int32 sums of
+// a whole K range stay in tensor memory -- no partial sums ever cross shared
+// memory.  The A operand is read from tensor memory too: unpack warps expand the
+// 2-bit weights to unsigned bytes in registers (one shift-and-mask per four
+// weights) and write them with tcgen05.st, so the expanded weights never touch
+// shared memory either.  What crosses shared memory is the packed stream (once in
+// by bulk copy, once out by 128-bit loads) and the tokens' codes (TMA).
 //
-// Weights are stored as u = w + 1 and fed as unsigned bytes, so the MMA computes
-// sum_k u*q = sum_k w*q + sum_k q; the per-token code sum is subtracted in the
-// epilogue (exact in int32).
+//   warp 0        producer: per 128-column block one bulk copy of a 4 KiB packed tile
+//                 and one TMA load of the codes [T_pad x 128], 16-stage ring
+//   warp 1        allocates tensor memory; one lane issues four MMAs per block
+//   warps 4..11   unpack: two groups of four warps (one per TMEM lane quadrant) take
+//                 alternate blocks into a ring of eight A buffers (32 columns each)
+//   warps 12..15  epilogue: read the accumulators (two D buffers alternate), subtract
+//                 the code sum (weights are fed as u = w + 1), rescale, store bf16
 //
-// A CTA owns 128 weight rows x Kc columns.  When K is split over several CTAs
-// the partial sums are combined with integer atomics (associative, so the
-// result does not depend on arrival order) into a zeroed scratch array and the
-// last CTA to arrive for a row group runs the epilogue.
-#include "hbl_common.cuh"
+// Work is dealt stream-K style: all (row block, column block) pairs in row-major
+// order, cut into equal contiguous ranges, one per CTA, so every SM streams the
+// same number of bytes.  A row block whose range is cut belongs to the CTA that
+// holds its first column block; the other CTAs write their partial sums to a slot
+// of their own in `part`, raise a flag, and the owner adds them when its own range
+// is done.  A CTA publishes before it ever waits, so the waits cannot cycle; every
+// wait is bounded and reports HBL_ERR_TIMEOUT.
+#include <cuda.h>
+
+#include "hbl_pipeline.cuh"
 
 namespace hbl {
 namespace {
 
-constexpr int kWarps = 4;
-constexpr int kSlabsPerWarp = 2;
-constexpr int kRowsPerCta = kWarps * kSlabsPerWarp * 16;   // 128
-constexpr int kDepth = 4;                                  // k-blocks of weights in flight per lane
+using namespace pipe;
 
-__device__ __forceinline__ void mma_u8s8(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+constexpr int THREADS = 512;
+constexpr int SW = 16;                 // shared-memory stages (packed tile + codes)
+constexpr int NA = 8;                  // A buffers in tensor memory
+constexpr int A_COL0 = 128;            // D buffers: columns [0,64) and [64,128); A buffers from column 128
+constexpr int TMEM_COLS = 512;
+constexpr int TILE_BYTES = 4096;       // 128 rows x 128 columns x 2 bits
+constexpr int MAX_GRID = 160;
+
+struct Params {
+  const float* scale; const int32_t* codesum; const unsigned char* Wp; const float* alpha;
+  __nv_bfloat16* y; int32_t* acc_out;
+  int32_t* part;      // [grid][t_pad][128] partial sums of row blocks this CTA does not own
+  int* flags;         // [grid], zero on entry
+  int* status;
+  int T, K, N, t_pad;
+};
+
+// Instruction descriptor: D s32 (2 << 4), A unsigned 8-bit (0 << 7), B signed 8-bit (1 << 10),
+// both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+__device__ __forceinline__ uint32_t make_idesc(int n_tok) {
+  return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n_tok >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+// Shared-memory matrix descriptor, K-major, 128-byte swizzle, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-      : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void umma_i8_tmem_a(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
 }
 
-// NT = number of 8-token MMA tiles (padded tokens = 8*NT).
-template <int NT>
-__global__ void __launch_bounds__(kWarps * 32)
-gemm_stream_kernel(const int8_t* __restrict__ codes, const float* __restrict__ scale,
-                   const int32_t* __restrict__ codesum, int T, int K, int Kc,
-                   const uint4* __restrict__ Wp, int N, const float* __restrict__ alpha,
-                   __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out,
-                   int32_t* __restrict__ acc_ws, int* __restrict__ counters) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ int s_is_last;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, t4 = lane & 3;
-  const int splits = K / Kc;
-  const int rg = blockIdx.x / splits;            // row group
-  const int sp = blockIdx.x % splits;            // k split
-  const int k0 = sp * Kc;
-  const int ctiles = K / 128;
-  const int nkb = Kc / 128;
-  const int stride = Kc + 16;                    // bytes per staged token row
-  constexpr int TP = 8 * NT;
-
-  // ---- start the weight stream before anything else ----
-  const int rt0 = rg * (kRowsPerCta / 16) + warp * kSlabsPerWarp;
-  const int n_rt = N / 16;
-  const uint4* wsrc[kSlabsPerWarp];
-  bool slab_ok[kSlabsPerWarp];
-#pragma unroll
-  for (int s = 0; s < kSlabsPerWarp; ++s) {
-    slab_ok[s] = (rt0 + s) < n_rt;
-    wsrc[s] = Wp + ((size_t)(slab_ok[s] ? rt0 + s : 0) * ctiles + k0 / 128) * 32 + lane;
+// One contiguous piece of a CTA's range: column blocks [ka, ke) of row block rb.
+struct Segment { int rb, ka, ke; };
+struct Range {
+  long u0, u1;
+  int n_kb;
+  long pos;
+  __device__ Range(long u0_, long u1_, int n_kb_) : u0(u0_), u1(u1_), n_kb(n_kb_), pos(u0_) {}
+  __device__ bool next(Segment& s) {
+    if (pos >= u1) return false;
+    s.rb = (int)(pos / n_kb);
+    s.ka = (int)(pos % n_kb);
+    const long end = (long)(s.rb + 1) * n_kb;
+    s.ke = (int)((u1 < end ? u1 : end) - (long)s.rb * n_kb);
+    pos = (long)s.rb * n_kb + s.ke;
+    return true;
   }
-  uint4 ring[kDepth][kSlabsPerWarp];
-#pragma unroll
-  for (int d = 0; d < kDepth; ++d)
-#pragma unroll
-    for (int s = 0; s < kSlabsPerWarp; ++s)
-      ring[d][s] = (d < nkb && slab_ok[s]) ? __ldcs(wsrc[s] + (size_t)d * 32) : make_uint4(0, 0, 0, 0);
+};
 
-  // ---- stage this CTA's slice of the codes: [TP][Kc] bytes, rows >= T zero ----
-  {
-    const int vec_per_row = Kc / 16;
-    for (int i = tid; i < TP * vec_per_row; i += kWarps * 32) {
-      const int r = i / vec_per_row, c = i % vec_per_row;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (r < T) v = *reinterpret_cast<const uint4*>(codes + (size_t)r * K + k0 + c * 16);
-      *reinterpret_cast<uint4*>(smem_raw + (size_t)r * stride + c * 16) = v;
-    }
+template <int T_PAD>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p) {
+  constexpr int STAGE_BYTES = TILE_BYTES + T_PAD * 128;
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) uint64_t w_full[SW], w_empty[SW], a_full[NA], a_empty[NA], d_full[2], d_empty[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+  unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_kb = p.K / 128, n_rb = (p.N + 127) / 128;
+  const long U = (long)n_rb * n_kb;
+  const int G = gridDim.x, c = blockIdx.x;
+  const long u0 = U * c / G, u1 = U * (c + 1) / G;
+
+  if (tid == 0) {
+    for (int s = 0; s < SW; ++s) { mbar_init(&w_full[s], 1); mbar_init(&w_empty[s], 1); }
+    for (int a = 0; a < NA; ++a) { mbar_init(&a_full[a], 4); mbar_init(&a_empty[a], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&d_full[b], 1); mbar_init(&d_empty[b], 4); }
+    abort_flag_s = 0;
+    mbar_fence_init();
   }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                 "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
 
-  int acc[kSlabsPerWarp][NT][4];
-#pragma unroll
-  for (int s = 0; s < kSlabsPerWarp; ++s)
-#pragma unroll
-    for (int n = 0; n < NT; ++n)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) acc[s][n][i] = 0;
-
-  const unsigned char* brow = smem_raw + (size_t)g * stride + 4 * t4;
-  for (int kb0 = 0; kb0 < nkb; kb0 += kDepth) {
-#pragma unroll
-    for (int d = 0; d < kDepth; ++d) {
-      const int kb = kb0 + d;
-      if (kb < nkb) {
-        uint4 cur[kSlabsPerWarp];
-#pragma unroll
-        for (int s = 0; s < kSlabsPerWarp; ++s) {
-          cur[s] = ring[d][s];
-          if (kb + kDepth < nkb && slab_ok[s]) ring[d][s] = __ldcs(wsrc[s] + (size_t)(kb + kDepth) * 32);
+  if (warp == 0) {
+    // ------------------------------ producer ------------------------------
+    if (lane == 0) {
+      Range range(u0, u1, n_kb);
+      Segment sg;
+      uint32_t i = 0;
+      bool ok = true;
+      while (ok && range.next(sg)) {
+        for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
+          const int s = i % SW;
+          if (!mbar_wait(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+          unsigned char* st = stages + (size_t)s * STAGE_BYTES;
+          mbar_expect_tx(&w_full[s], STAGE_BYTES);
+          bulk_load(st, p.Wp + ((size_t)sg.rb * n_kb + kb) * TILE_BYTES, TILE_BYTES, &w_full[s]);
+          tma_load_2d(st + TILE_BYTES, &tm_codes, &w_full[s], kb * 128, 0);
         }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(T_PAD);
+      Range range(u0, u1, n_kb);
+      Segment sg;
+      uint32_t i = 0, seg = 0;
+      bool ok = true;
+      while (ok && range.next(sg)) {
+        const int b = seg & 1;
+        if (!mbar_wait(&d_empty[b], ((seg >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)b * 64;
+        for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
+          const int s = i % SW, a = i % NA;
+          if (!mbar_wait(&w_full[s], (i / SW) & 1, abort_flag, p.status)) { ok = false; break; }     // the codes have landed
+          if (!mbar_wait(&a_full[a], (i / NA) & 1, abort_flag, p.status)) { ok = false; break; }     // the weights are in tensor memory
+          tc_fence_after();
+          const uint64_t bdesc = make_desc(smem_u32(stages + (size_t)s * STAGE_BYTES + TILE_BYTES));
+          const uint32_t a_tmem = tmem_base + A_COL0 + 32u * a;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint32_t b0[NT], b1[NT];
+          for (int ks = 0; ks < 4; ++ks)
+            umma_i8_tmem_a(d_tmem, a_tmem + 8u * ks, bdesc + (uint64_t)(2 * ks), idesc, (kb > sg.ka) || ks > 0);
+          umma_commit(&w_empty[s]);          // the stage's codes have been read
+          umma_commit(&a_empty[a]);          // and so has the A buffer
+        }
+        if (ok) umma_commit(&d_full[b]);
+        ++seg;
+      }
+    }
+  } else if (warp >= 4 && warp < 12) {
+    // ------------------------------ unpack ------------------------------
+    const int group = (warp - 4) >> 2, quad = warp & 3;
+    const int row = quad * 32 + lane;
+    Range range(u0, u1, n_kb);
+    Segment sg;
+    uint32_t i = 0;
+    bool ok = true;
+    while (ok && range.next(sg)) {
+      for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
+        if ((int)(i & 1) != group) continue;
+        const int s = i % SW, a = i % NA;
+        ok = mbar_wait(&w_full[s], (i / SW) & 1, abort_flag, p.status) &&
+             mbar_wait(&a_empty[a], ((i / NA) & 1) ^ 1, abort_flag, p.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const unsigned char* st = stages + (size_t)s * STAGE_BYTES;
+        const uint4 lo = *reinterpret_cast<const uint4*>(st + row * 16);
+        const uint4 hi = *reinterpret_cast<const uint4*>(st + 2048 + row * 16);
+        const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+        uint32_t r[32];
 #pragma unroll
-          for (int n = 0; n < NT; ++n) {
-            const unsigned char* p = brow + (size_t)n * 8 * stride + kb * 128 + j * 32;
-            b0[n] = *reinterpret_cast<const uint32_t*>(p);
-            b1[n] = *reinterpret_cast<const uint32_t*>(p + 16);
+        for (int kq = 0; kq < 8; ++kq)
+#pragma unroll
+          for (int q = 0; q < 4; ++q) r[kq * 4 + q] = (w[kq] >> (2 * q)) & 0x03030303u;   // column kq*4+q: k = 16 kq + 4 q + byte
+        tmem_st32(tmem_base + A_COL0 + 32u * a + ((uint32_t)(quad * 32) << 16), r);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&a_full[a]);
+      }
+    }
+  } else if (warp >= 12) {
+    // ------------------------------ epilogue ------------------------------
+    const int quad = warp & 3;
+    const int row_in_block = quad * 32 + lane;
+    const float al = (p.acc_out == nullptr) ? __ldg(p.alpha) : 0.f;
+    auto finish = [&](int rb, const int (&v)[T_PAD]) {
+      const int row = rb * 128 + row_in_block;
+      if (row >= p.N) return;
+#pragma unroll
+      for (int t = 0; t < T_PAD; ++t) {
+        if (t >= p.T) break;
+        const int a = v[t] - __ldg(p.codesum + t);
+        if (p.acc_out != nullptr) p.acc_out[(size_t)t * p.N + row] = a;
+        else p.y[(size_t)t * p.N + row] = __float2bfloat16_rn((float)a * (__ldg(p.scale + t) * al));
+      }
+    };
+    Range range(u0, u1, n_kb);
+    Segment sg;
+    uint32_t seg = 0;
+    bool ok = true;
+    int own[T_PAD];               // sums of the row block this CTA owns but does not complete (its last segment)
+    int own_rb = -1;
+    while (range.next(sg)) {
+      const int b = seg & 1;
+      ok = ok && mbar_wait(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      int v[T_PAD];
+      if (ok) {
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < T_PAD / 16; ++j) {
+          uint32_t r[16];
+          tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 64 + j * 16), r);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int t = 0; t < 16; ++t) v[j * 16 + t] = (int)r[t];
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&d_empty[b]);
+      }
+      ++seg;
+      const bool whole = sg.ka == 0 && sg.ke == n_kb;
+      if (sg.ka != 0) {
+        // not the owner: publish the partial sums ([t][128 rows], coalesced), then raise this CTA's flag
+        if (ok) {
+#pragma unroll
+          for (int t = 0; t < T_PAD; ++t) __stcg(p.part + ((size_t)c * T_PAD + t) * 128 + row_in_block, v[t]);
+          __threadfence();
+        }
+        named_barrier(3, 128);                                // all four epilogue warps have written
+        if (ok && warp == 12 && lane == 0) atomicExch(p.flags + c, 1);
+      } else if (whole) {
+        if (ok) finish(sg.rb, v);
+      } else if (ok) {
+#pragma unroll
+        for (int t = 0; t < T_PAD; ++t) own[t] = v[t];
+        own_rb = sg.rb;
+      }
+    }
+    if (own_rb >= 0 && ok) {
+      // the row block continues in the next CTAs: collect their parts (each was published before its CTA waits for anything)
+      const long end = (long)(own_rb + 1) * n_kb;
+      for (int f = c + 1; f < G && U * f / G < end && ok; ++f) {
+        int ready = 0;
+        if (lane == 0) {
+          volatile int* flag = p.flags + f;
+          const uint64_t t0 = global_ns();
+          while (!(ready = *flag)) {
+            if (*abort_flag) break;
+            if (global_ns() - t0 > 2000000000ull) {
+              report_device_error(p.status, HBL_ERR_TIMEOUT);
+              *abort_flag = 1;
+              break;
+            }
+            __nanosleep(64);
           }
-#pragma unroll
-          for (int s = 0; s < kSlabsPerWarp; ++s) {
-            const uint32_t w = (j == 0) ? cur[s].x : (j == 1) ? cur[s].y : (j == 2) ? cur[s].z : cur[s].w;
-            uint32_t a[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) a[i] = (w >> (2 * i)) & 0x03030303u;
-#pragma unroll
-            for (int n = 0; n < NT; ++n) mma_u8s8(acc[s][n], a, b0[n], b1[n]);
-          }
         }
+        ok = __shfl_sync(0xffffffffu, ready, 0) != 0;
+        if (!ok) break;
+        __threadfence();
+#pragma unroll
+        for (int t = 0; t < T_PAD; ++t) own[t] += __ldcg(p.part + ((size_t)f * T_PAD + t) * 128 + row_in_block);
       }
+      if (ok) finish(own_rb, own);
     }
   }
 
-  // ---- combine / epilogue ----
-  // Fragment element i of acc[s][n]: weight row rbase + g + 8*(i>>1), token 8n + 2*t4 + (i&1).
-  const bool direct = (splits == 1);
-  if (direct) {
-    const float al = (acc_out == nullptr) ? __ldg(alpha) : 0.f;
-#pragma unroll
-    for (int n = 0; n < NT; ++n)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int tok = 8 * n + 2 * t4 + (i & 1);
-        if (tok >= T) continue;
-        const int cs = __ldg(codesum + tok);
-        const float f = (acc_out == nullptr) ? __ldg(scale + tok) * al : 0.f;
-#pragma unroll
-        for (int s = 0; s < kSlabsPerWarp; ++s) {
-          if (!slab_ok[s]) continue;
-          const int row = (rt0 + s) * 16 + g + 8 * (i >> 1);
-          const int a = acc[s][n][i] - cs;
-          if (acc_out != nullptr) acc_out[(size_t)tok * N + row] = a;
-          else y[(size_t)tok * N + row] = __float2bfloat16_rn((float)a * f);
-        }
-      }
-    return;
+  // ------------------------------ teardown ------------------------------
+  __syncwarp();
+  if (*abort_flag) {
+    // give copies that are still in flight time to land before the CTA's shared memory goes away
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) __nanosleep(1000);
   }
-#pragma unroll
-  for (int n = 0; n < NT; ++n)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int tok = 8 * n + 2 * t4 + (i & 1);
-      if (tok >= T) continue;
-#pragma unroll
-      for (int s = 0; s < kSlabsPerWarp; ++s) {
-        if (!slab_ok[s]) continue;
-        const int row = (rt0 + s) * 16 + g + 8 * (i >> 1);
-        atomicAdd(acc_ws + (size_t)tok * N + row, acc[s][n][i]);
-      }
-    }
-  __threadfence();
+  tc_fence_before();
   __syncthreads();
-  if (tid == 0) s_is_last = (atomicAdd(counters + rg, 1) == splits - 1);
-  __syncthreads();
-  if (!s_is_last) return;
-  __threadfence();
-  {
-    const float al = (acc_out == nullptr) ? __ldg(alpha) : 0.f;
-    const int row_base = rg * kRowsPerCta;
-    const int rows = min(kRowsPerCta, N - row_base);
-    for (int i = tid; i < T * rows; i += kWarps * 32) {
-      const int tok = i / rows, row = row_base + i % rows;
-      const int a = __ldcg(acc_ws + (size_t)tok * N + row) - __ldg(codesum + tok);
-      if (acc_out != nullptr) acc_out[(size_t)tok * N + row] = a;
-      else y[(size_t)tok * N + row] = __float2bfloat16_rn((float)a * (__ldg(scale + tok) * al));
-    }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
-int choose_kc(int N, int K, int max_kc) {
-  const int row_groups = (N + kRowsPerCta - 1) / kRowsPerCta;
-  const int cands[5] = {2048, 1024, 512, 256, 128};
-  int smallest = 128;
-  for (int i = 0; i < 5; ++i) {
-    if (cands[i] > max_kc || K % cands[i] != 0) continue;
-    smallest = cands[i];
-    if ((long)row_groups * (K / cands[i]) >= 148L * 3) return cands[i];
+// ---- host side ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
   }
-  return smallest;
+  return fn;
 }
 
-template <int NT>
-int launch_nt(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
-              const void* Wp, int N, const float* alpha, __nv_bfloat16* y, int32_t* acc_out,
-              int32_t* acc_ws, int* counters, cudaStream_t s) {
-  const int Kc = choose_kc(N, K, NT <= 2 ? 2048 : (NT == 4 ? 1024 : 512));   // staged codes stay <= 33 KiB
-  const int splits = K / Kc;
-  const int row_groups = (N + kRowsPerCta - 1) / kRowsPerCta;
-  const size_t smem = (size_t)8 * NT * (Kc + 16);
-  auto kern = gemm_stream_kernel<NT>;
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+int pad_tokens(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
+
+template <int T_PAD>
+int launch_variant(const CUtensorMap& tm, const Params& p, int grid, cudaStream_t s) {
+  constexpr size_t smem = (size_t)SW * (TILE_BYTES + T_PAD * 128) + 1024;
+  auto kern = gemm_stream_kernel<T_PAD>;
+  static bool done = false;   // idempotent attribute; a race only repeats the call
+  if (!done) {
+    HBL_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    done = true;
+  }
   profile_before(KERNEL_CONTRACT, s);
-  kern<<<row_groups * splits, kWarps * 32, smem, s>>>(codes, scale, codesum, T, K, Kc,
-                                                      static_cast<const uint4*>(Wp), N, alpha, y, acc_out,
-                                                      acc_ws, counters);
+  kern<<<grid, THREADS, smem, s>>>(tm, p);
   profile_after(KERNEL_CONTRACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -215,20 +387,43 @@ int launch_nt(const int8_t* codes, const float* scale, const int32_t* codesum, i
 
 }  // namespace
 
-size_t gemm_stream_acc_words(int T, int N) { return (size_t)T * N; }
-size_t gemm_stream_counter_words(int N) { return (size_t)(N + kRowsPerCta - 1) / kRowsPerCta; }
+// Scratch of the streaming contraction: `part` slots (contents irrelevant on entry) and flags (zero on entry).
+size_t gemm_stream_acc_words(int T, int N) { (void)N; return (size_t)MAX_GRID * 128 * pad_tokens(T < 1 ? 1 : T); }
+size_t gemm_stream_counter_words(int N) { (void)N; return MAX_GRID; }
 
-// acc_ws [T*N] and counters must be zero on entry when K is split (the caller
-// clears them; the activation kernel does it as a side job in hbl_forward).
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
                        const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s) {
   if (T <= 0) return HBL_OK;
   if (T > 64) return HBL_ERR_TOO_LARGE;
-  if (T <= 8) return launch_nt<1>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
-  if (T <= 16) return launch_nt<2>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
-  if (T <= 32) return launch_nt<4>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
-  return launch_nt<8>(codes, scale, codesum, T, K, W_packed, N, alpha, y, acc_out, acc_ws, counters, s);
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return HBL_ERR_CUDA;
+  const int t_pad = pad_tokens(T);
+  CUtensorMap tm;
+  {
+    // codes [T, K] int8 row-major; box = 128 bytes of K x t_pad tokens (rows beyond T read as zero), 128-byte swizzle
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)T};
+    cuuint64_t strides[1] = {(cuuint64_t)K};
+    cuuint32_t box[2] = {128u, (cuuint32_t)t_pad};
+    cuuint32_t estr[2] = {1, 1};
+    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(codes), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return HBL_ERR_CUDA;
+  }
+  Params p;
+  p.scale = scale; p.codesum = codesum; p.Wp = static_cast<const unsigned char*>(W_packed); p.alpha = alpha;
+  p.y = y; p.acc_out = acc_out; p.part = acc_ws; p.flags = counters;
+  p.status = device_status_word();
+  if (p.status == nullptr) return HBL_ERR_CUDA;
+  p.T = T; p.K = K; p.N = N; p.t_pad = t_pad;
+  const long U = (long)((N + 127) / 128) * (K / 128);
+  int grid = sm_count();
+  if (grid > MAX_GRID) grid = MAX_GRID;
+  if (U < grid) grid = (int)U;
+  if (t_pad == 16) return launch_variant<16>(tm, p, grid, s);
+  if (t_pad == 32) return launch_variant<32>(tm, p, grid, s);
+  return launch_variant<64>(tm, p, grid, s);
 }
 
 }  // namespace hbl

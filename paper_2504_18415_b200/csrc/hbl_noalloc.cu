@@ -1,15 +1,16 @@
 // hbl_gemm_i32_static: the streaming contraction kernel for callers that cannot
-// provide (or allocate) a workspace.  Its split-K scratch -- the int32 partial
-// sums and the per-row-group arrival counters -- lives in a fixed array inside
-// the library's device image instead of in caller memory.
+// provide (or allocate) a workspace.  Its scratch -- the slots in which CTAs hand
+// partial sums of a shared row block to the block's owner, and the flags that say
+// a slot is complete -- lives in a fixed array inside the library's device image
+// instead of in caller memory.
 #include "hbl_common.cuh"
 
 using namespace hbl;
 
 namespace {
 
-constexpr size_t kStaticAccWords = 262144;      // tokens * out_dim may not exceed this (1 MiB of int32)
-constexpr size_t kStaticCounterWords = 1024;    // row groups of 128 outputs: out_dim <= 131072
+constexpr size_t kStaticAccWords = 160 * 128 * 16;   // one 128-row x 16-token slot of partial sums per CTA (1.25 MiB): tokens <= 16
+constexpr size_t kStaticCounterWords = 256;          // one flag per CTA
 constexpr size_t kStaticScratchBytes = (kStaticAccWords + kStaticCounterWords) * sizeof(int32_t);
 
 // Every GPU that loads the library holds this array until the process exits.

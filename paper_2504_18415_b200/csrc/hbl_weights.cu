@@ -1,13 +1,15 @@
 // Weight side of H-BitLinear: the per-tensor absmean ternary quantizer (Eq. 1-2)
 // and the 2-bit storage format.
 //
-// Format (also described in hbl.h): W[N,K] is cut into tiles of 16 rows x 128
-// columns; a tile is 512 bytes = 32 "lanes" x four 32-bit words.  Word j of
-// lane l carries the 16 weights that lane l of a warp feeds to one
-// m16n8k32 integer MMA as its A fragment (four 8-bit x4 registers a0..a3):
-//   a_i byte b  =  W[16*rt + (l>>2) + 8*(i&1)][128*ct + 32*j + 16*(i>>1) + 4*(l&3) + b]
-// stored as u = w + 1 (0,1,2) at bit 8*b + 2*i, so that (word >> 2*i) & 0x03030303
-// is register a_i, ready to use as four unsigned bytes.
+// Format (also described in hbl.h): W[N,K] is cut into tiles of 128 rows x 128
+// columns (rows padded with zeros up to a multiple of 128), 4096 bytes each,
+// ordered [row block][column block].  A tile is [h = 0,1][row 0..127][four 32-bit
+// words]: word v of (h, row) holds the 16 weights of that row in columns
+// 16*(4h+v) .. +15 of the tile, column 4*i + b at bit 8*b + 2*i, stored as
+// u = w + 1 (0,1,2).  So (word >> 2*i) & 0x03030303 is four consecutive weights of
+// one row as unsigned bytes -- what a thread that owns one row of a tensor-memory
+// operand needs -- and a thread reads its row's 32 bytes with two conflict-free
+// 128-bit shared-memory loads.
 #include "hbl_common.cuh"
 
 namespace hbl {
@@ -51,11 +53,11 @@ absmean_partial_kernel(const void* __restrict__ W, int is_bf16, size_t total, do
 }
 
 // Pass 2: every CTA re-derives alpha from the partials (fixed order), then
-// ternarises and packs.  One thread = one (tile, lane) = four packed words.
+// ternarises and packs.  One thread = one packed word = 16 weights of one row.
 __global__ void __launch_bounds__(256)
 ternarise_pack_kernel(const void* __restrict__ W, int is_bf16, int N, int K, float eps,
                       const double* __restrict__ partials, int n_partials,
-                      uint4* __restrict__ packed, float* __restrict__ alpha_out) {
+                      uint32_t* __restrict__ packed, float* __restrict__ alpha_out) {
   __shared__ float s_alpha;
   if (threadIdx.x == 0) {
     double t = 0.0;
@@ -66,60 +68,49 @@ ternarise_pack_kernel(const void* __restrict__ W, int is_bf16, int N, int K, flo
   }
   __syncthreads();
   const float d = s_alpha + eps;
-  const int ctiles = K / 128;
-  const size_t n_items = (size_t)(N / 16) * ctiles * 32;
-  for (size_t it = (size_t)blockIdx.x * 256 + threadIdx.x; it < n_items; it += (size_t)gridDim.x * 256) {
-    const int l = (int)(it & 31);
-    const size_t tile = it >> 5;
-    const int ct = (int)(tile % ctiles);
-    const int rt = (int)(tile / ctiles);
-    const int row0 = rt * 16 + (l >> 2);
-    const int col0 = ct * 128 + 4 * (l & 3);
-    uint32_t words[4];
+  const int n_kb = K / 128;
+  const size_t n_words = (size_t)((N + 127) / 128) * n_kb * 1024;
+  for (size_t it = (size_t)blockIdx.x * 256 + threadIdx.x; it < n_words; it += (size_t)gridDim.x * 256) {
+    const int v = (int)(it & 3), row = (int)((it >> 2) & 127), h = (int)((it >> 9) & 1);
+    const size_t tile = it >> 10;
+    const int kb = (int)(tile % n_kb), rb = (int)(tile / n_kb);
+    const int R = rb * 128 + row;
+    uint32_t wd = 0x55555555u;                                // padding rows: w = 0
+    if (R < N) {
+      wd = 0;
+      const size_t base = (size_t)R * K + (size_t)kb * 128 + 16 * (4 * h + v);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t wd = 0;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const size_t base = (size_t)(row0 + 8 * (i & 1)) * K + col0 + 32 * j + 16 * (i >> 1);
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
-          const float w = load_w(W, is_bf16, base + b);
+          const float w = load_w(W, is_bf16, base + 4 * i + b);
           float r = rintf(__fdiv_rn(w, d));                 // round half to even
           r = fminf(fmaxf(r, -1.0f), 1.0f);
           wd |= (uint32_t)((int)r + 1) << (8 * b + 2 * i);
         }
-      }
-      words[j] = wd;
     }
-    packed[it] = make_uint4(words[0], words[1], words[2], words[3]);
+    packed[it] = wd;
   }
 }
 
-// Packed -> int8 [N,K] row-major (values -1,0,1).  One thread = one (tile, lane).
+// Packed -> int8 [N,K] row-major (values -1,0,1).  One thread = one packed word = 16 weights of one row.
 __global__ void __launch_bounds__(256)
-unpack_kernel(const uint4* __restrict__ packed, int N, int K, int8_t* __restrict__ out) {
-  const int ctiles = K / 128;
-  const size_t n_items = (size_t)(N / 16) * ctiles * 32;
-  for (size_t it = (size_t)blockIdx.x * 256 + threadIdx.x; it < n_items; it += (size_t)gridDim.x * 256) {
-    const int l = (int)(it & 31);
-    const size_t tile = it >> 5;
-    const int ct = (int)(tile % ctiles);
-    const int rt = (int)(tile / ctiles);
-    const int row0 = rt * 16 + (l >> 2);
-    const int col0 = ct * 128 + 4 * (l & 3);
-    const uint4 q = __ldg(packed + it);
-    const uint32_t words[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t u = (words[j] >> (2 * i)) & 0x03030303u;   // four bytes in {0,1,2}
-        const uint32_t s = __vsub4(u, 0x01010101u);               // per-byte w = u - 1
-        const size_t base = (size_t)(row0 + 8 * (i & 1)) * K + col0 + 32 * j + 16 * (i >> 1);
-        *reinterpret_cast<uint32_t*>(out + base) = s;
-      }
-    }
+unpack_kernel(const uint32_t* __restrict__ packed, int N, int K, int8_t* __restrict__ out) {
+  const int n_kb = K / 128;
+  const size_t n_words = (size_t)((N + 127) / 128) * n_kb * 1024;
+  for (size_t it = (size_t)blockIdx.x * 256 + threadIdx.x; it < n_words; it += (size_t)gridDim.x * 256) {
+    const int v = (int)(it & 3), row = (int)((it >> 2) & 127), h = (int)((it >> 9) & 1);
+    const size_t tile = it >> 10;
+    const int kb = (int)(tile % n_kb), rb = (int)(tile / n_kb);
+    const int R = rb * 128 + row;
+    if (R >= N) continue;
+    const uint32_t wd = __ldg(packed + it);
+    uint4 o;
+    o.x = __vsub4(wd & 0x03030303u, 0x01010101u);            // per-byte w = u - 1: columns 0..3 of the 16
+    o.y = __vsub4((wd >> 2) & 0x03030303u, 0x01010101u);
+    o.z = __vsub4((wd >> 4) & 0x03030303u, 0x01010101u);
+    o.w = __vsub4((wd >> 6) & 0x03030303u, 0x01010101u);
+    *reinterpret_cast<uint4*>(out + (size_t)R * K + (size_t)kb * 128 + 16 * (4 * h + v)) = o;
   }
 }
 
@@ -134,20 +125,20 @@ int launch_weight_quant(const void* W, int w_dtype, int N, int K, float eps, voi
   absmean_partial_kernel<<<grid, kReduceThreads, 0, s>>>(W, w_dtype == HBL_BF16, total, partials);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
-  const size_t n_items = total / 16;
-  int grid2 = (int)min((size_t)148 * 16, (n_items + 255) / 256);
+  const size_t n_words = (size_t)((N + 127) / 128) * (K / 128) * 1024;
+  int grid2 = (int)min((size_t)148 * 16, (n_words + 255) / 256);
   ternarise_pack_kernel<<<grid2, 256, 0, s>>>(W, w_dtype == HBL_BF16, N, K, eps, partials, grid,
-                                              static_cast<uint4*>(packed), alpha);
+                                              static_cast<uint32_t*>(packed), alpha);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
 }
 
 int launch_unpack_weights(const void* packed, int N, int K, int8_t* out, cudaStream_t s) {
-  const size_t n_items = (size_t)N * K / 16;
-  int grid = (int)min((size_t)148 * 16, (n_items + 255) / 256);
+  const size_t n_words = (size_t)((N + 127) / 128) * (K / 128) * 1024;
+  int grid = (int)min((size_t)148 * 16, (n_words + 255) / 256);
   profile_before(KERNEL_UNPACK, s);
-  unpack_kernel<<<grid, 256, 0, s>>>(static_cast<const uint4*>(packed), N, K, out);
+  unpack_kernel<<<grid, 256, 0, s>>>(static_cast<const uint32_t*>(packed), N, K, out);
   profile_after(KERNEL_UNPACK, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());

@@ -29,20 +29,25 @@ def test_packed_format_is_the_documented_one():
     N, K = 32, 256
     W = wl.rows("latent", 3, 77, K, 0, N, "f32")
     packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), EPS)
-    words = packed.cpu().numpy().view(np.uint32).reshape(N // 16, K // 128, 32, 4)
+    words = packed.cpu().numpy().view(np.uint32).reshape((N + 127) // 128, K // 128, 2, 128, 4)
     wt, _ = orc.weight_quant(W, EPS, 32)
     dec = np.zeros((N, K), np.int8)
-    for rt in range(N // 16):
-        for ct in range(K // 128):
-            for l in range(32):
-                for j in range(4):
-                    w = int(words[rt, ct, l, j])
-                    for i in range(4):
-                        for b in range(4):
-                            u = (w >> (8 * b + 2 * i)) & 3
-                            dec[16 * rt + (l >> 2) + 8 * (i & 1), 128 * ct + 32 * j + 16 * (i >> 1) + 4 * (l & 3) + b] = u - 1
+    for rb in range(words.shape[0]):
+        for kb in range(K // 128):
+            for h in range(2):
+                for row in range(128):
+                    R = 128 * rb + row
+                    for v in range(4):
+                        w = int(words[rb, kb, h, row, v])
+                        for i in range(4):
+                            for b in range(4):
+                                u = (w >> (8 * b + 2 * i)) & 3
+                                if R < N:
+                                    dec[R, 128 * kb + 16 * (4 * h + v) + 4 * i + b] = u - 1
+                                else:
+                                    assert u == 1          # padding rows are zeros
     assert np.array_equal(dec, wt)
-    assert packed.numel() == N * K // 4
+    assert packed.numel() == ((N + 127) // 128) * 128 * K // 4
 
 
 def test_weight_quant_special_values():

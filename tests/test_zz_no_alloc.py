@@ -33,8 +33,8 @@ def _problem(T, K, N, bits, seed):
 
 @pytest.mark.gpu
 def test_static_scratch_matches_workspace_version_on_consecutive_calls():
-    # split-K shapes (scratch is really used), a ragged token count, then a smaller problem that
-    # would see the first one's partial sums if the array were not cleared
+    # shapes whose row blocks are shared between thread blocks (scratch is really used), a ragged token
+    # count, then a smaller problem that would trip over the first one's flags if they were not cleared
     shapes = [(16, 8192, 2048, 4), (5, 4096, 528, 8), (16, 8192, 2048, 4), (1, 2048, 2048, 4)]
     for n, (T, K, N, bits) in enumerate(shapes):
         q, csum, packed = _problem(T, K, N, bits, 700 + n)
@@ -59,8 +59,8 @@ def test_sizes_beyond_the_fixed_array_are_refused_on_the_host():
     p, n = C.c_void_p(1024), C.c_void_p(0)
     call = lambda T, K, N: L.hbl_gemm_i32_static(p, p, T, K, p, N, p, n)
     assert call(65, 1024, 1024) == 11          # beyond the streaming kernel's token limit
-    assert call(64, 1024, 8192) == 11          # 64 * 8192 > 262144 scratch words
-    assert call(16, 1024, 32768) == 11
-    assert call(16, 65536, 1024) == 11
+    assert call(64, 1024, 8192) == 11          # the fixed array holds slots for 16 tokens
+    assert call(17, 1024, 1024) == 11
+    assert call(16, 65536, 1024) == 11         # in_dim beyond the library's maximum
     assert call(16, 1000, 1024) == 2           # shape errors still come first
     assert call(0, 1024, 1024) == 0            # nothing to do
