@@ -36,9 +36,10 @@ namespace {
 using namespace pipe;
 
 constexpr int THREADS = 512;
-constexpr int SW = 16;                 // shared-memory stages (packed tile + codes)
-constexpr int NA = 8;                  // A buffers in tensor memory
+constexpr int MAX_SW = 12;             // shared-memory stages (packed tiles + codes of one unit)
+constexpr int MAX_NA = 12;             // A buffers in tensor memory
 constexpr int A_COL0 = 128;            // D buffers: columns [0,64) and [64,128); A buffers from column 128
+constexpr int SMEM_RING_BYTES = 192 * 1024;
 constexpr int TMEM_COLS = 512;
 constexpr int TILE_BYTES = 4096;       // 128 rows x 128 columns x 2 bits
 constexpr int MAX_GRID = 160;
@@ -119,19 +120,31 @@ struct Range {
   }
 };
 
-template <int T_PAD>
+// A unit of work is KBP consecutive 128-column blocks of one row block: the single MMA-issuing
+// thread pays one barrier wait and two commits per unit, so wider units keep it ahead of the stream.
+template <int T_PAD, int KBP>
+struct Geo {
+  static constexpr int STAGE_BYTES = KBP * (TILE_BYTES + T_PAD * 128);
+  static constexpr int SW_RAW = SMEM_RING_BYTES / STAGE_BYTES;
+  static constexpr int SW = SW_RAW > MAX_SW ? MAX_SW : SW_RAW;
+  static constexpr int NA = (TMEM_COLS - A_COL0) / (32 * KBP);
+  static constexpr int CODES_OFF = KBP * TILE_BYTES;
+};
+
+template <int T_PAD, int KBP>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p) {
-  constexpr int STAGE_BYTES = TILE_BYTES + T_PAD * 128;
+  using GEO = Geo<T_PAD, KBP>;
+  constexpr int STAGE_BYTES = GEO::STAGE_BYTES, SW = GEO::SW, NA = GEO::NA;
   extern __shared__ unsigned char smem_dyn[];
-  __shared__ __align__(8) uint64_t w_full[SW], w_empty[SW], a_full[NA], a_empty[NA], d_full[2], d_empty[2];
+  __shared__ __align__(8) uint64_t w_full[MAX_SW], w_empty[MAX_SW], a_full[MAX_NA], a_empty[MAX_NA], d_full[2], d_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
   unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_kb = p.K / 128, n_rb = (p.N + 127) / 128;
+  const int n_kb = p.K / (128 * KBP), n_rb = (p.N + 127) / 128;   // units per row block
   const long U = (long)n_rb * n_kb;
   const int G = gridDim.x, c = blockIdx.x;
   const long u0 = U * c / G, u1 = U * (c + 1) / G;
@@ -166,8 +179,10 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
           if (!mbar_wait(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
           unsigned char* st = stages + (size_t)s * STAGE_BYTES;
           mbar_expect_tx(&w_full[s], STAGE_BYTES);
-          bulk_load(st, p.Wp + ((size_t)sg.rb * n_kb + kb) * TILE_BYTES, TILE_BYTES, &w_full[s]);
-          tma_load_2d(st + TILE_BYTES, &tm_codes, &w_full[s], kb * 128, 0);
+          bulk_load(st, p.Wp + ((size_t)sg.rb * n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[s]);
+#pragma unroll
+          for (int j = 0; j < KBP; ++j)
+            tma_load_2d(st + GEO::CODES_OFF + j * (T_PAD * 128), &tm_codes, &w_full[s], (kb * KBP + j) * 128, 0);
         }
       }
     }
@@ -186,14 +201,20 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
         const uint32_t d_tmem = tmem_base + (uint32_t)b * 64;
         for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
           const int s = i % SW, a = i % NA;
-          if (!mbar_wait(&w_full[s], (i / SW) & 1, abort_flag, p.status)) { ok = false; break; }     // the codes have landed
-          if (!mbar_wait(&a_full[a], (i / NA) & 1, abort_flag, p.status)) { ok = false; break; }     // the weights are in tensor memory
+          // The unpack warps waited for the stage (weights and codes) before they filled the A buffer,
+          // so one wait covers both operands.
+          if (!mbar_wait(&a_full[a], (i / NA) & 1, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t bdesc = make_desc(smem_u32(stages + (size_t)s * STAGE_BYTES + TILE_BYTES));
-          const uint32_t a_tmem = tmem_base + A_COL0 + 32u * a;
+          const uint32_t codes_sm = smem_u32(stages + (size_t)s * STAGE_BYTES + GEO::CODES_OFF);
+          const uint32_t a_tmem = tmem_base + A_COL0 + (uint32_t)(32 * KBP) * a;
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            umma_i8_tmem_a(d_tmem, a_tmem + 8u * ks, bdesc + (uint64_t)(2 * ks), idesc, (kb > sg.ka) || ks > 0);
+          for (int j = 0; j < KBP; ++j) {
+            const uint64_t bdesc = make_desc(codes_sm + j * (T_PAD * 128));
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              umma_i8_tmem_a(d_tmem, a_tmem + 32u * j + 8u * ks, bdesc + (uint64_t)(2 * ks), idesc,
+                             (kb > sg.ka) || j > 0 || ks > 0);
+          }
           umma_commit(&w_empty[s]);          // the stage's codes have been read
           umma_commit(&a_empty[a]);          // and so has the A buffer
         }
@@ -219,15 +240,18 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
         if (!ok) break;
         tc_fence_after();
         const unsigned char* st = stages + (size_t)s * STAGE_BYTES;
-        const uint4 lo = *reinterpret_cast<const uint4*>(st + row * 16);
-        const uint4 hi = *reinterpret_cast<const uint4*>(st + 2048 + row * 16);
-        const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-        uint32_t r[32];
 #pragma unroll
-        for (int kq = 0; kq < 8; ++kq)
+        for (int j = 0; j < KBP; ++j) {
+          const uint4 lo = *reinterpret_cast<const uint4*>(st + j * TILE_BYTES + row * 16);
+          const uint4 hi = *reinterpret_cast<const uint4*>(st + j * TILE_BYTES + 2048 + row * 16);
+          const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+          uint32_t r[32];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) r[kq * 4 + q] = (w[kq] >> (2 * q)) & 0x03030303u;   // column kq*4+q: k = 16 kq + 4 q + byte
-        tmem_st32(tmem_base + A_COL0 + 32u * a + ((uint32_t)(quad * 32) << 16), r);
+          for (int kq = 0; kq < 8; ++kq)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) r[kq * 4 + q] = (w[kq] >> (2 * q)) & 0x03030303u;   // column kq*4+q: k = 16 kq + 4 q + byte
+          tmem_st32(tmem_base + A_COL0 + (uint32_t)(32 * KBP) * a + 32u * j + ((uint32_t)(quad * 32) << 16), r);
+        }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         tc_fence_before();
         __syncwarp();
@@ -297,26 +321,55 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
     if (own_rb >= 0 && ok) {
       // the row block continues in the next CTAs: collect their parts (each was published before its CTA waits for anything)
       const long end = (long)(own_rb + 1) * n_kb;
-      for (int f = c + 1; f < G && U * f / G < end && ok; ++f) {
-        int ready = 0;
-        if (lane == 0) {
-          volatile int* flag = p.flags + f;
+      int n_follow = 0;
+      while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < end) ++n_follow;
+      // wait for all of them at once: lane l polls the flags of followers l, l+32, ...
+      {
+        int ready = 1;
+        for (int f = lane; f < n_follow && ready; f += 32) {
+          volatile int* flag = p.flags + c + 1 + f;
           const uint64_t t0 = global_ns();
-          while (!(ready = *flag)) {
-            if (*abort_flag) break;
+          while (!*flag) {
+            if (*abort_flag) { ready = 0; break; }
             if (global_ns() - t0 > 2000000000ull) {
               report_device_error(p.status, HBL_ERR_TIMEOUT);
               *abort_flag = 1;
+              ready = 0;
               break;
             }
             __nanosleep(64);
           }
         }
-        ok = __shfl_sync(0xffffffffu, ready, 0) != 0;
-        if (!ok) break;
+        ok = __all_sync(0xffffffffu, ready);
+      }
+      if (ok) {
         __threadfence();
+        // independent loads, four followers in flight at a time
+        for (int f0 = 0; f0 < n_follow; f0 += 4) {
+          int tmp[4][T_PAD <= 16 ? T_PAD : 1];
+          if constexpr (T_PAD <= 16) {
 #pragma unroll
-        for (int t = 0; t < T_PAD; ++t) own[t] += __ldcg(p.part + ((size_t)f * T_PAD + t) * 128 + row_in_block);
+            for (int j = 0; j < 4; ++j) {
+              const int f = f0 + j < n_follow ? f0 + j : n_follow - 1;
+#pragma unroll
+              for (int t = 0; t < T_PAD; ++t)
+                tmp[j][t] = __ldcg(p.part + ((size_t)(c + 1 + f) * T_PAD + t) * 128 + row_in_block);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (f0 + j < n_follow) {
+#pragma unroll
+                for (int t = 0; t < T_PAD; ++t) own[t] += tmp[j][t];
+              }
+          } else {
+            (void)tmp;
+            for (int j = 0; j < 4 && f0 + j < n_follow; ++j) {
+#pragma unroll
+              for (int t = 0; t < T_PAD; ++t)
+                own[t] += __ldcg(p.part + ((size_t)(c + 1 + f0 + j) * T_PAD + t) * 128 + row_in_block);
+            }
+          }
+        }
       }
       if (ok) finish(own_rb, own);
     }
@@ -368,10 +421,11 @@ int sm_count() {
 
 int pad_tokens(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
 
-template <int T_PAD>
+template <int T_PAD, int KBP>
 int launch_variant(const CUtensorMap& tm, const Params& p, int grid, cudaStream_t s) {
-  constexpr size_t smem = (size_t)SW * (TILE_BYTES + T_PAD * 128) + 1024;
-  auto kern = gemm_stream_kernel<T_PAD>;
+  using GEO = Geo<T_PAD, KBP>;
+  constexpr size_t smem = (size_t)GEO::SW * GEO::STAGE_BYTES + 1024;
+  auto kern = gemm_stream_kernel<T_PAD, KBP>;
   static bool done = false;   // idempotent attribute; a race only repeats the call
   if (!done) {
     HBL_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -383,6 +437,13 @@ int launch_variant(const CUtensorMap& tm, const Params& p, int grid, cudaStream_
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
+}
+
+template <int T_PAD>
+int launch_kbp(int kbp, const CUtensorMap& tm, const Params& p, int grid, cudaStream_t s) {
+  if (kbp == 4) return launch_variant<T_PAD, 4>(tm, p, grid, s);
+  if (kbp == 2) return launch_variant<T_PAD, 2>(tm, p, grid, s);
+  return launch_variant<T_PAD, 1>(tm, p, grid, s);
 }
 
 }  // namespace
@@ -417,13 +478,17 @@ int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* c
   p.status = device_status_word();
   if (p.status == nullptr) return HBL_ERR_CUDA;
   p.T = T; p.K = K; p.N = N; p.t_pad = t_pad;
-  const long U = (long)((N + 127) / 128) * (K / 128);
-  int grid = sm_count();
-  if (grid > MAX_GRID) grid = MAX_GRID;
-  if (U < grid) grid = (int)U;
-  if (t_pad == 16) return launch_variant<16>(tm, p, grid, s);
-  if (t_pad == 32) return launch_variant<32>(tm, p, grid, s);
-  return launch_variant<64>(tm, p, grid, s);
+  int n_sm = sm_count();
+  if (n_sm > MAX_GRID) n_sm = MAX_GRID;
+  // Column blocks per unit: as wide as K allows while every CTA still gets a few units.
+  const long blocks = (long)((N + 127) / 128) * (K / 128);
+  int kbp = 4;
+  while (kbp > 1 && ((K / 128) % kbp != 0 || blocks / kbp < 4L * n_sm)) kbp >>= 1;
+  const long U = blocks / kbp;
+  const int grid = (int)(U < n_sm ? U : n_sm);
+  if (t_pad == 16) return launch_kbp<16>(kbp, tm, p, grid, s);
+  if (t_pad == 32) return launch_kbp<32>(kbp, tm, p, grid, s);
+  return launch_kbp<64>(kbp, tm, p, grid, s);
 }
 
 }  // namespace hbl
