@@ -131,6 +131,7 @@ act_quant_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int bits, f
   __shared__ float red_f[32];
   __shared__ int red_i[TPC];
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a programmatic dependent may start; it waits before reading our output
   const int tid_cta = threadIdx.x;
   // side job: clear the caller's scratch words (split-K accumulators of the next kernel)
   if (zero_fill != nullptr) {
@@ -298,6 +299,7 @@ act_quant_generic_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int
                          size_t zero_words) {
   __shared__ float red_f[8];
   __shared__ int red_i[8];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (zero_fill != nullptr)
     for (size_t i = (size_t)blockIdx.x * 256 + tid; i < zero_words; i += (size_t)gridDim.x * 256)

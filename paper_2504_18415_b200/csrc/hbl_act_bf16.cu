@@ -144,6 +144,9 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   __shared__ float red_f[THREADS / 32];
   __shared__ int red_i[THREADS / 32];
 
+  // A kernel launched as a programmatic dependent of this one may start now; it waits
+  // (griddepcontrol.wait) before it touches anything written here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int tid_cta = threadIdx.x;
   if (zero_fill != nullptr) {   // side job: clear the caller's scratch words
     for (size_t i = (size_t)blockIdx.x * THREADS + tid_cta; i < zero_words; i += (size_t)gridDim.x * THREADS)

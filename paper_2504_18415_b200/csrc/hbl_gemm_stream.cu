@@ -80,6 +80,9 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
+// Returns once the kernel this one depends on has completed and its writes are visible
+// (immediately when the launch was an ordinary one).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -169,6 +172,22 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
   if (warp == 0) {
     // ------------------------------ producer ------------------------------
     if (lane == 0) {
+      // The packed weights do not depend on the kernel that quantizes the activations: when this
+      // kernel was launched early (programmatic dependent launch) the first ring-full of weight
+      // copies is in flight before that kernel has finished.  The codes are fetched after the wait.
+      uint32_t primed = 0;
+      {
+        Range range(u0, u1, n_kb);
+        Segment sg;
+        while (primed < (uint32_t)SW && range.next(sg)) {
+          for (int kb = sg.ka; kb < sg.ke && primed < (uint32_t)SW; ++kb, ++primed) {
+            mbar_expect_tx(&w_full[primed], STAGE_BYTES);
+            bulk_load(stages + (size_t)primed * STAGE_BYTES, p.Wp + ((size_t)sg.rb * n_kb + kb) * (KBP * TILE_BYTES),
+                      KBP * TILE_BYTES, &w_full[primed]);
+          }
+        }
+      }
+      grid_dependency_wait();
       Range range(u0, u1, n_kb);
       Segment sg;
       uint32_t i = 0;
@@ -176,10 +195,12 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
       while (ok && range.next(sg)) {
         for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
           const int s = i % SW;
-          if (!mbar_wait(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
           unsigned char* st = stages + (size_t)s * STAGE_BYTES;
-          mbar_expect_tx(&w_full[s], STAGE_BYTES);
-          bulk_load(st, p.Wp + ((size_t)sg.rb * n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[s]);
+          if (i >= primed) {
+            if (!mbar_wait(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+            mbar_expect_tx(&w_full[s], STAGE_BYTES);
+            bulk_load(st, p.Wp + ((size_t)sg.rb * n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[s]);
+          }
 #pragma unroll
           for (int j = 0; j < KBP; ++j)
             tma_load_2d(st + GEO::CODES_OFF + j * (T_PAD * 128), &tm_codes, &w_full[s], (kb * KBP + j) * 128, 0);
@@ -260,6 +281,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
     }
   } else if (warp >= 12) {
     // ------------------------------ epilogue ------------------------------
+    grid_dependency_wait();                                  // scales, code sums and cleared flags come from the previous kernel
     const int quad = warp & 3;
     const int row_in_block = quad * 32 + lane;
     const float al = (p.acc_out == nullptr) ? __ldg(p.alpha) : 0.f;
@@ -431,8 +453,20 @@ int launch_variant(const CUtensorMap& tm, const Params& p, int grid, cudaStream_
     HBL_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     done = true;
   }
+  // Programmatic dependent launch: if the previous operation on the stream is a kernel that signals
+  // griddepcontrol.launch_dependents (the activation kernels do), this kernel may start while it runs.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   profile_before(KERNEL_CONTRACT, s);
-  kern<<<grid, THREADS, smem, s>>>(tm, p);
+  HBL_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, tm, p));
   profile_after(KERNEL_CONTRACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
