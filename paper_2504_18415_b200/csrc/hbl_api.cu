@@ -261,6 +261,18 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   }
   const int src[7] = {0, 0, 0, 1, 2, 2, 3};                  // which quantized input feeds each projection
   const int out_dims[7] = {H, H, H, H, F, F, H};
+  if (stream_path) {
+    // small batch: all seven weight tensors stream through one launch
+    StreamInput inputs[4];
+    for (int i = 0; i < 4; ++i)
+      inputs[i] = {reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
+                   reinterpret_cast<int32_t*>(ws + w.codesum[i]), in_dims[i]};
+    StreamJob jobs[7];
+    for (int i = 0; i < 7; ++i)
+      jobs[i] = {Ws[i], b->alpha7 + i, static_cast<__nv_bfloat16*>(ys[i]), nullptr, out_dims[i], src[i]};
+    return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, reinterpret_cast<int32_t*>(ws + w.acc[0]),
+                                    reinterpret_cast<int*>(ws + w.counters[0]), s);
+  }
   for (int i = 0; i < 7; ++i) {
     const int xi = src[i];
     rc = run_gemm(p, reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]),

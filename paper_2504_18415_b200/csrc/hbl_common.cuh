@@ -59,6 +59,11 @@ int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* c
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s);
 int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
                        const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s);
+// Several weight tensors, each reading one of up to four quantized inputs, in one launch (T <= 64).
+struct StreamInput { const int8_t* codes; const float* scale; const int32_t* codesum; int K; };
+struct StreamJob { const void* W_packed; const float* alpha; __nv_bfloat16* y; int32_t* acc_out; int N; int input; };
+int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
+                             int32_t* part, int* flags, cudaStream_t s);
 size_t gemm_stream_acc_words(int T, int N);       // int32 words of split-K scratch (0 if none)
 size_t gemm_stream_counter_words(int N);
 

@@ -44,14 +44,27 @@ constexpr int TMEM_COLS = 512;
 constexpr int TILE_BYTES = 4096;       // 128 rows x 128 columns x 2 bits
 constexpr int MAX_GRID = 160;
 
-struct Params {
-  const float* scale; const int32_t* codesum; const unsigned char* Wp; const float* alpha;
+constexpr int MAX_JOBS = 8;            // weight tensors contracted by one launch (a decoder block has seven)
+constexpr int MAX_MAPS = 4;            // distinct quantized inputs they read (a decoder block has four)
+
+// One weight tensor and where its result goes.  Units (KBP column blocks of one row block) are
+// numbered across all jobs of a launch: this job's are [u_begin, u_begin + n_rb * n_kb).
+struct Job {
+  const unsigned char* Wp; const float* scale; const int32_t* codesum; const float* alpha;
   __nv_bfloat16* y; int32_t* acc_out;
+  int N, n_kb, map;
+  long u_begin;
+};
+struct Params {
+  Job jobs[MAX_JOBS];
+  int n_jobs;
+  long U;             // units of all jobs
   int32_t* part;      // [grid][t_pad][128] partial sums of row blocks this CTA does not own
   int* flags;         // [grid], zero on entry
   int* status;
-  int T, K, N, t_pad;
+  int T;
 };
+struct CodeMaps { CUtensorMap m[MAX_MAPS]; };   // codes [T, K] of each input, box 128 x T_pad, 128-byte swizzle
 
 // Instruction descriptor: D s32 (2 << 4), A unsigned 8-bit (0 << 7), B signed 8-bit (1 << 10),
 // both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
@@ -105,20 +118,24 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "memory");
 }
 
-// One contiguous piece of a CTA's range: column blocks [ka, ke) of row block rb.
-struct Segment { int rb, ka, ke; };
+// One contiguous piece of a CTA's range: units [ka, ke) of row block rb of one job.
+struct Segment { int job, rb, ka, ke; long rb_end; /* global index one past the row block's last unit */ };
 struct Range {
-  long u0, u1;
-  int n_kb;
-  long pos;
-  __device__ Range(long u0_, long u1_, int n_kb_) : u0(u0_), u1(u1_), n_kb(n_kb_), pos(u0_) {}
+  const Params& p;
+  long u1, pos;
+  __device__ Range(const Params& p_, long u0_, long u1_) : p(p_), u1(u1_), pos(u0_) {}
   __device__ bool next(Segment& s) {
     if (pos >= u1) return false;
-    s.rb = (int)(pos / n_kb);
-    s.ka = (int)(pos % n_kb);
-    const long end = (long)(s.rb + 1) * n_kb;
-    s.ke = (int)((u1 < end ? u1 : end) - (long)s.rb * n_kb);
-    pos = (long)s.rb * n_kb + s.ke;
+    int j = 0;
+    while (j + 1 < p.n_jobs && pos >= p.jobs[j + 1].u_begin) ++j;
+    const long local = pos - p.jobs[j].u_begin;
+    const int n_kb = p.jobs[j].n_kb;
+    s.job = j;
+    s.rb = (int)(local / n_kb);
+    s.ka = (int)(local % n_kb);
+    s.rb_end = p.jobs[j].u_begin + (long)(s.rb + 1) * n_kb;
+    s.ke = (int)((u1 < s.rb_end ? u1 : s.rb_end) - (s.rb_end - n_kb));
+    pos = s.rb_end - n_kb + s.ke;
     return true;
   }
 };
@@ -136,7 +153,7 @@ struct Geo {
 
 template <int T_PAD, int KBP>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p) {
+gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant__ Params p) {
   using GEO = Geo<T_PAD, KBP>;
   constexpr int STAGE_BYTES = GEO::STAGE_BYTES, SW = GEO::SW, NA = GEO::NA;
   extern __shared__ unsigned char smem_dyn[];
@@ -147,8 +164,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
   unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_kb = p.K / (128 * KBP), n_rb = (p.N + 127) / 128;   // units per row block
-  const long U = (long)n_rb * n_kb;
+  const long U = p.U;
   const int G = gridDim.x, c = blockIdx.x;
   const long u0 = U * c / G, u1 = U * (c + 1) / G;
 
@@ -177,33 +193,36 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
       // copies is in flight before that kernel has finished.  The codes are fetched after the wait.
       uint32_t primed = 0;
       {
-        Range range(u0, u1, n_kb);
+        Range range(p, u0, u1);
         Segment sg;
         while (primed < (uint32_t)SW && range.next(sg)) {
+          const Job& job = p.jobs[sg.job];
           for (int kb = sg.ka; kb < sg.ke && primed < (uint32_t)SW; ++kb, ++primed) {
             mbar_expect_tx(&w_full[primed], STAGE_BYTES);
-            bulk_load(stages + (size_t)primed * STAGE_BYTES, p.Wp + ((size_t)sg.rb * n_kb + kb) * (KBP * TILE_BYTES),
-                      KBP * TILE_BYTES, &w_full[primed]);
+            bulk_load(stages + (size_t)primed * STAGE_BYTES,
+                      job.Wp + ((size_t)sg.rb * job.n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[primed]);
           }
         }
       }
       grid_dependency_wait();
-      Range range(u0, u1, n_kb);
+      Range range(p, u0, u1);
       Segment sg;
       uint32_t i = 0;
       bool ok = true;
       while (ok && range.next(sg)) {
+        const Job& job = p.jobs[sg.job];
+        const CUtensorMap* tm_codes = &maps.m[job.map];
         for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
           const int s = i % SW;
           unsigned char* st = stages + (size_t)s * STAGE_BYTES;
           if (i >= primed) {
             if (!mbar_wait(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
             mbar_expect_tx(&w_full[s], STAGE_BYTES);
-            bulk_load(st, p.Wp + ((size_t)sg.rb * n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[s]);
+            bulk_load(st, job.Wp + ((size_t)sg.rb * job.n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[s]);
           }
 #pragma unroll
           for (int j = 0; j < KBP; ++j)
-            tma_load_2d(st + GEO::CODES_OFF + j * (T_PAD * 128), &tm_codes, &w_full[s], (kb * KBP + j) * 128, 0);
+            tma_load_2d(st + GEO::CODES_OFF + j * (T_PAD * 128), tm_codes, &w_full[s], (kb * KBP + j) * 128, 0);
         }
       }
     }
@@ -211,7 +230,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
       const uint32_t idesc = make_idesc(T_PAD);
-      Range range(u0, u1, n_kb);
+      Range range(p, u0, u1);
       Segment sg;
       uint32_t i = 0, seg = 0;
       bool ok = true;
@@ -247,7 +266,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
     // ------------------------------ unpack ------------------------------
     const int group = (warp - 4) >> 2, quad = warp & 3;
     const int row = quad * 32 + lane;
-    Range range(u0, u1, n_kb);
+    Range range(p, u0, u1);
     Segment sg;
     uint32_t i = 0;
     bool ok = true;
@@ -284,24 +303,26 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
     grid_dependency_wait();                                  // scales, code sums and cleared flags come from the previous kernel
     const int quad = warp & 3;
     const int row_in_block = quad * 32 + lane;
-    const float al = (p.acc_out == nullptr) ? __ldg(p.alpha) : 0.f;
-    auto finish = [&](int rb, const int (&v)[T_PAD]) {
+    auto finish = [&](int job_idx, int rb, const int (&v)[T_PAD]) {
+      const Job& job = p.jobs[job_idx];
       const int row = rb * 128 + row_in_block;
-      if (row >= p.N) return;
+      if (row >= job.N) return;
+      const float al = (job.acc_out == nullptr) ? __ldg(job.alpha) : 0.f;
 #pragma unroll
       for (int t = 0; t < T_PAD; ++t) {
         if (t >= p.T) break;
-        const int a = v[t] - __ldg(p.codesum + t);
-        if (p.acc_out != nullptr) p.acc_out[(size_t)t * p.N + row] = a;
-        else p.y[(size_t)t * p.N + row] = __float2bfloat16_rn((float)a * (__ldg(p.scale + t) * al));
+        const int a = v[t] - __ldg(job.codesum + t);
+        if (job.acc_out != nullptr) job.acc_out[(size_t)t * job.N + row] = a;
+        else job.y[(size_t)t * job.N + row] = __float2bfloat16_rn((float)a * (__ldg(job.scale + t) * al));
       }
     };
-    Range range(u0, u1, n_kb);
+    Range range(p, u0, u1);
     Segment sg;
     uint32_t seg = 0;
     bool ok = true;
     int own[T_PAD];               // sums of the row block this CTA owns but does not complete (its last segment)
-    int own_rb = -1;
+    int own_rb = -1, own_job = 0;
+    long own_end = 0;
     while (range.next(sg)) {
       const int b = seg & 1;
       ok = ok && mbar_wait(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
@@ -322,7 +343,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
         if (lane == 0) mbar_arrive(&d_empty[b]);
       }
       ++seg;
-      const bool whole = sg.ka == 0 && sg.ke == n_kb;
+      const bool whole = sg.ka == 0 && sg.ke == p.jobs[sg.job].n_kb;
       if (sg.ka != 0) {
         // not the owner: publish the partial sums ([t][128 rows], coalesced), then raise this CTA's flag
         if (ok) {
@@ -333,16 +354,18 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
         named_barrier(3, 128);                                // all four epilogue warps have written
         if (ok && warp == 12 && lane == 0) atomicExch(p.flags + c, 1);
       } else if (whole) {
-        if (ok) finish(sg.rb, v);
+        if (ok) finish(sg.job, sg.rb, v);
       } else if (ok) {
 #pragma unroll
         for (int t = 0; t < T_PAD; ++t) own[t] = v[t];
         own_rb = sg.rb;
+        own_job = sg.job;
+        own_end = sg.rb_end;
       }
     }
     if (own_rb >= 0 && ok) {
       // the row block continues in the next CTAs: collect their parts (each was published before its CTA waits for anything)
-      const long end = (long)(own_rb + 1) * n_kb;
+      const long end = own_end;
       int n_follow = 0;
       while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < end) ++n_follow;
       // wait for all of them at once: lane l polls the flags of followers l, l+32, ...
@@ -393,7 +416,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tm_codes, const Params p)
           }
         }
       }
-      if (ok) finish(own_rb, own);
+      if (ok) finish(own_job, own_rb, own);
     }
   }
 
@@ -444,7 +467,7 @@ int sm_count() {
 int pad_tokens(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
 
 template <int T_PAD, int KBP>
-int launch_variant(const CUtensorMap& tm, const Params& p, int grid, cudaStream_t s) {
+int launch_variant(const CodeMaps& maps, const Params& p, int grid, cudaStream_t s) {
   using GEO = Geo<T_PAD, KBP>;
   constexpr size_t smem = (size_t)GEO::SW * GEO::STAGE_BYTES + 1024;
   auto kern = gemm_stream_kernel<T_PAD, KBP>;
@@ -466,7 +489,7 @@ int launch_variant(const CUtensorMap& tm, const Params& p, int grid, cudaStream_
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   profile_before(KERNEL_CONTRACT, s);
-  HBL_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, tm, p));
+  HBL_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, maps, p));
   profile_after(KERNEL_CONTRACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -474,10 +497,10 @@ int launch_variant(const CUtensorMap& tm, const Params& p, int grid, cudaStream_
 }
 
 template <int T_PAD>
-int launch_kbp(int kbp, const CUtensorMap& tm, const Params& p, int grid, cudaStream_t s) {
-  if (kbp == 4) return launch_variant<T_PAD, 4>(tm, p, grid, s);
-  if (kbp == 2) return launch_variant<T_PAD, 2>(tm, p, grid, s);
-  return launch_variant<T_PAD, 1>(tm, p, grid, s);
+int launch_kbp(int kbp, const CodeMaps& maps, const Params& p, int grid, cudaStream_t s) {
+  if (kbp == 4) return launch_variant<T_PAD, 4>(maps, p, grid, s);
+  if (kbp == 2) return launch_variant<T_PAD, 2>(maps, p, grid, s);
+  return launch_variant<T_PAD, 1>(maps, p, grid, s);
 }
 
 }  // namespace
@@ -486,43 +509,71 @@ int launch_kbp(int kbp, const CUtensorMap& tm, const Params& p, int grid, cudaSt
 size_t gemm_stream_acc_words(int T, int N) { (void)N; return (size_t)MAX_GRID * 128 * pad_tokens(T < 1 ? 1 : T); }
 size_t gemm_stream_counter_words(int N) { (void)N; return MAX_GRID; }
 
-int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
-                       const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
-                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s) {
-  if (T <= 0) return HBL_OK;
+// Several weight tensors (each reading one of up to four quantized inputs) in one launch.
+int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
+                             int32_t* part, int* flags, cudaStream_t s) {
+  if (T <= 0 || n_jobs <= 0) return HBL_OK;
   if (T > 64) return HBL_ERR_TOO_LARGE;
+  if (n_jobs > MAX_JOBS || n_inputs > MAX_MAPS || n_inputs <= 0) return HBL_ERR_SHAPE;
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return HBL_ERR_CUDA;
   const int t_pad = pad_tokens(T);
-  CUtensorMap tm;
-  {
+  CodeMaps maps;
+  for (int m = 0; m < MAX_MAPS; ++m) {
     // codes [T, K] int8 row-major; box = 128 bytes of K x t_pad tokens (rows beyond T read as zero), 128-byte swizzle
-    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)T};
-    cuuint64_t strides[1] = {(cuuint64_t)K};
+    const StreamInput& in = inputs[m < n_inputs ? m : 0];
+    cuuint64_t dims[2] = {(cuuint64_t)in.K, (cuuint64_t)T};
+    cuuint64_t strides[1] = {(cuuint64_t)in.K};
     cuuint32_t box[2] = {128u, (cuuint32_t)t_pad};
     cuuint32_t estr[2] = {1, 1};
-    if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(codes), dims, strides, box, estr,
+    if (fn(&maps.m[m], CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(in.codes), dims, strides, box, estr,
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return HBL_ERR_CUDA;
   }
-  Params p;
-  p.scale = scale; p.codesum = codesum; p.Wp = static_cast<const unsigned char*>(W_packed); p.alpha = alpha;
-  p.y = y; p.acc_out = acc_out; p.part = acc_ws; p.flags = counters;
-  p.status = device_status_word();
-  if (p.status == nullptr) return HBL_ERR_CUDA;
-  p.T = T; p.K = K; p.N = N; p.t_pad = t_pad;
   int n_sm = sm_count();
   if (n_sm > MAX_GRID) n_sm = MAX_GRID;
-  // Column blocks per unit: as wide as K allows while every CTA still gets a few units.
-  const long blocks = (long)((N + 127) / 128) * (K / 128);
+  // Column blocks per unit: as wide as every K allows while every CTA still gets a few units.
+  long blocks = 0;
+  for (int j = 0; j < n_jobs; ++j) blocks += (long)((jobs[j].N + 127) / 128) * (inputs[jobs[j].input].K / 128);
   int kbp = 4;
-  while (kbp > 1 && ((K / 128) % kbp != 0 || blocks / kbp < 4L * n_sm)) kbp >>= 1;
-  const long U = blocks / kbp;
-  const int grid = (int)(U < n_sm ? U : n_sm);
-  if (t_pad == 16) return launch_kbp<16>(kbp, tm, p, grid, s);
-  if (t_pad == 32) return launch_kbp<32>(kbp, tm, p, grid, s);
-  return launch_kbp<64>(kbp, tm, p, grid, s);
+  for (;;) {
+    bool fits = blocks / kbp >= 4L * n_sm;
+    for (int m = 0; m < n_inputs; ++m) fits = fits && (inputs[m].K / 128) % kbp == 0;
+    if (fits || kbp == 1) break;
+    kbp >>= 1;
+  }
+  Params p;
+  p.n_jobs = n_jobs;
+  long u = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    const StreamInput& in = inputs[jobs[j].input];
+    Job& jb = p.jobs[j];
+    jb.Wp = static_cast<const unsigned char*>(jobs[j].W_packed);
+    jb.scale = in.scale; jb.codesum = in.codesum; jb.alpha = jobs[j].alpha;
+    jb.y = jobs[j].y; jb.acc_out = jobs[j].acc_out;
+    jb.N = jobs[j].N; jb.n_kb = in.K / (128 * kbp); jb.map = jobs[j].input;
+    jb.u_begin = u;
+    u += (long)((jobs[j].N + 127) / 128) * jb.n_kb;
+  }
+  for (int j = n_jobs; j < MAX_JOBS; ++j) p.jobs[j] = p.jobs[0];
+  p.U = u;
+  p.part = part; p.flags = flags;
+  p.status = device_status_word();
+  if (p.status == nullptr) return HBL_ERR_CUDA;
+  p.T = T;
+  const int grid = (int)(u < n_sm ? u : n_sm);
+  if (t_pad == 16) return launch_kbp<16>(kbp, maps, p, grid, s);
+  if (t_pad == 32) return launch_kbp<32>(kbp, maps, p, grid, s);
+  return launch_kbp<64>(kbp, maps, p, grid, s);
+}
+
+int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
+                       const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
+                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s) {
+  StreamInput in = {codes, scale, codesum, K};
+  StreamJob job = {W_packed, alpha, y, acc_out, N, 0};
+  return launch_gemm_stream_multi(&in, 1, &job, 1, T, acc_ws, counters, s);
 }
 
 }  // namespace hbl
