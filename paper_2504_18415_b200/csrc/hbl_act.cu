@@ -131,7 +131,7 @@ act_quant_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int bits, f
   __shared__ float red_f[32];
   __shared__ int red_i[TPC];
 
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a programmatic dependent may start; it waits before reading our output
+  grid_launch_dependents();   // a programmatic dependent may start; it waits before reading our output
   const int tid_cta = threadIdx.x;
   // side job: clear the caller's scratch words (split-K accumulators of the next kernel)
   if (zero_fill != nullptr) {
@@ -288,6 +288,7 @@ act_quant_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int bits, f
     scale[token] = __fdiv_rn(st, c);
     if (codesum != nullptr) codesum[token] = csum;
   }
+  grid_dependency_wait();   // chain: this kernel is complete only when the one before it is
 }
 
 // No transform and K not a power of two: a plain two-pass kernel, one CTA per
@@ -299,7 +300,7 @@ act_quant_generic_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int
                          size_t zero_words) {
   __shared__ float red_f[8];
   __shared__ int red_i[8];
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  grid_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (zero_fill != nullptr)
     for (size_t i = (size_t)blockIdx.x * 256 + tid; i < zero_words; i += (size_t)gridDim.x * 256)
@@ -355,6 +356,7 @@ act_quant_generic_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int
     scale[token] = __fdiv_rn(st, c);
     if (codesum != nullptr) codesum[token] = t;
   }
+  grid_dependency_wait();
 }
 
 template <int M, int E, bool HAD>
@@ -376,7 +378,8 @@ int launch_one(const void* x, int x_dtype, int T, int bits, float eps, int8_t* c
   }
   const int grid = (T + TPC - 1) / TPC;
   profile_before(KERNEL_ACT, s);
-  kern<<<grid, THREADS, smem, s>>>(x, x_dtype == HBL_BF16, T, bits, eps, codes, scale, codesum, xr_out, zf, zw);
+  HBL_CUDA_OK(launch_dependent(kern, dim3(grid), dim3(THREADS), smem, s, x, (int)(x_dtype == HBL_BF16), T, bits, eps,
+                               codes, scale, codesum, xr_out, zf, zw));
   profile_after(KERNEL_ACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -413,8 +416,8 @@ int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use
   if (use_hadamard) return HBL_ERR_NOT_POW2;
   if (xr_out != nullptr) return HBL_ERR_SHAPE;
   profile_before(KERNEL_ACT, s);
-  act_quant_generic_kernel<<<T, 256, 0, s>>>(x, x_dtype == HBL_BF16, T, K, bits, eps, codes, scale, codesum,
-                                             zero_fill, zero_fill_words);
+  HBL_CUDA_OK(launch_dependent(act_quant_generic_kernel, dim3(T), dim3(256), 0, s, x, (int)(x_dtype == HBL_BF16), T, K,
+                               bits, eps, codes, scale, codesum, zero_fill, zero_fill_words));
   profile_after(KERNEL_ACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());

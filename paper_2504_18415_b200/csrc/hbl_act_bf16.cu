@@ -146,7 +146,7 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
 
   // A kernel launched as a programmatic dependent of this one may start now; it waits
   // (griddepcontrol.wait) before it touches anything written here.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  grid_launch_dependents();
   const int tid_cta = threadIdx.x;
   if (zero_fill != nullptr) {   // side job: clear the caller's scratch words
     for (size_t i = (size_t)blockIdx.x * THREADS + tid_cta; i < zero_words; i += (size_t)gridDim.x * THREADS)
@@ -401,6 +401,7 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
     if (live && tid == 0) codesum[token] = csum;
   }
   if (live && tid == 0) scale[token] = __fdiv_rn(st, cq);
+  grid_dependency_wait();   // chain: this kernel is complete only when the one before it is
 }
 
 template <int M, int BITS>
@@ -418,8 +419,8 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
   }
   const int grid = (T + G::TPC - 1) / G::TPC;
   profile_before(KERNEL_ACT, s);
-  kern<<<grid, G::THREADS, smem, s>>>(static_cast<const __nv_bfloat16*>(x), T, eps, codes, scale, codesum, xr_out,
-                                      zf, zw);
+  HBL_CUDA_OK(launch_dependent(kern, dim3(grid), dim3(G::THREADS), smem, s, static_cast<const __nv_bfloat16*>(x), T, eps,
+                               codes, scale, codesum, xr_out, zf, zw));
   profile_after(KERNEL_ACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());

@@ -33,6 +33,30 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
     if (_e != cudaSuccess) return HBL_ERR_CUDA;   \
   } while (0)
 
+// ---- programmatic dependent launch ----------------------------------------------
+// A kernel launched with launch_dependent() may start while the kernel before it on the stream is
+// still running, provided that kernel executes griddepcontrol.launch_dependents (or has exited).
+// The dependent must call grid_dependency_wait() before it reads anything the earlier kernel
+// writes.  The activation kernels also call it last thing, so that "kernel k has completed"
+// implies "kernels before k have completed" along a chain of such launches.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- kernel launchers (one per .cu file) -------------------------------------
 // Activation side: Eq. 3-6.
 int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use_hadamard, float eps,

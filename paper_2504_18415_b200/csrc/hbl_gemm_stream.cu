@@ -93,9 +93,6 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-// Returns once the kernel this one depends on has completed and its writes are visible
-// (immediately when the launch was an ordinary one).
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -478,18 +475,8 @@ int launch_variant(const CodeMaps& maps, const Params& p, int grid, cudaStream_t
   }
   // Programmatic dependent launch: if the previous operation on the stream is a kernel that signals
   // griddepcontrol.launch_dependents (the activation kernels do), this kernel may start while it runs.
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
   profile_before(KERNEL_CONTRACT, s);
-  HBL_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, maps, p));
+  HBL_CUDA_OK(launch_dependent(kern, dim3((unsigned)grid), dim3(THREADS), smem, s, maps, p));
   profile_after(KERNEL_CONTRACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
