@@ -55,7 +55,7 @@ typedef enum { HBL_F32 = 0, HBL_BF16 = 1 } hbl_dtype_t;
 /* Which contraction kernel hbl_forward / hbl_gemm_i32 use. */
 typedef enum {
   HBL_PATH_AUTO = 0,       /* by token count */
-  HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers); tokens <= 64 */
+  HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers into tensor memory); tokens <= 128 */
   HBL_PATH_TENSOR = 2      /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
 } hbl_path_t;
 

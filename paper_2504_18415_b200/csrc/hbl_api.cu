@@ -43,7 +43,7 @@ void profile_after(int kernel_id, cudaStream_t s) {
 
 namespace {
 
-constexpr int kStreamMaxTokens = 64;
+constexpr int kStreamMaxTokens = 128;
 constexpr int kMaxInDim = 32768;
 
 struct ForwardWs {           // byte offsets inside the caller's workspace

@@ -1,4 +1,4 @@
-// Small-batch contraction of H-BitLinear (Eq. 7) for T <= 64 tokens, bound by the
+// Small-batch contraction of H-BitLinear (Eq. 7) for T <= 128 tokens, bound by the
 // stream of 2-bit packed weights out of HBM.
 //
 // The roles are swapped with respect to the large-batch kernel: 128 weight rows
@@ -38,7 +38,7 @@ using namespace pipe;
 constexpr int THREADS = 512;
 constexpr int MAX_SW = 12;             // shared-memory stages (packed tiles + codes of one unit)
 constexpr int MAX_NA = 12;             // A buffers in tensor memory
-constexpr int A_COL0 = 128;            // D buffers: columns [0,64) and [64,128); A buffers from column 128
+// Tensor memory: two D buffers of D_COLS columns each, then the A buffers.
 constexpr int SMEM_RING_BYTES = 192 * 1024;
 constexpr int TMEM_COLS = 512;
 constexpr int TILE_BYTES = 4096;       // 128 rows x 128 columns x 2 bits
@@ -144,7 +144,10 @@ struct Geo {
   static constexpr int STAGE_BYTES = KBP * (TILE_BYTES + T_PAD * 128);
   static constexpr int SW_RAW = SMEM_RING_BYTES / STAGE_BYTES;
   static constexpr int SW = SW_RAW > MAX_SW ? MAX_SW : SW_RAW;
-  static constexpr int NA = (TMEM_COLS - A_COL0) / (32 * KBP);
+  static constexpr int D_COLS = T_PAD < 64 ? 64 : T_PAD;          // columns of one accumulator buffer
+  static constexpr int A_COL0 = 2 * D_COLS;
+  static constexpr int NA_RAW = (TMEM_COLS - A_COL0) / (32 * KBP);
+  static constexpr int NA = NA_RAW > MAX_NA ? MAX_NA : NA_RAW;
   static constexpr int CODES_OFF = KBP * TILE_BYTES;
 };
 
@@ -152,7 +155,7 @@ template <int T_PAD, int KBP>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant__ Params p) {
   using GEO = Geo<T_PAD, KBP>;
-  constexpr int STAGE_BYTES = GEO::STAGE_BYTES, SW = GEO::SW, NA = GEO::NA;
+  constexpr int STAGE_BYTES = GEO::STAGE_BYTES, SW = GEO::SW, NA = GEO::NA, D_COLS = GEO::D_COLS, A_COL0 = GEO::A_COL0;
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) uint64_t w_full[MAX_SW], w_empty[MAX_SW], a_full[MAX_NA], a_empty[MAX_NA], d_full[2], d_empty[2];
   __shared__ uint32_t tmem_slot;
@@ -235,7 +238,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
         const int b = seg & 1;
         if (!mbar_wait(&d_empty[b], ((seg >> 1) & 1) ^ 1, abort_flag, p.status)) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)b * 64;
+        const uint32_t d_tmem = tmem_base + (uint32_t)(b * D_COLS);
         for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
           const int s = i % SW, a = i % NA;
           // The unpack warps waited for the stage (weights and codes) before they filled the A buffer,
@@ -297,77 +300,83 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     }
   } else if (warp >= 12) {
     // ------------------------------ epilogue ------------------------------
+    // Accumulators are handled 16 token columns at a time, so nothing here needs more than a few
+    // dozen registers whatever T_PAD is.
     grid_dependency_wait();                                  // scales, code sums and cleared flags come from the previous kernel
     const int quad = warp & 3;
     const int row_in_block = quad * 32 + lane;
-    auto finish = [&](int job_idx, int rb, const int (&v)[T_PAD]) {
+    const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
+    auto finish_chunk = [&](int job_idx, int rb, int j, const int (&v)[16]) {
       const Job& job = p.jobs[job_idx];
       const int row = rb * 128 + row_in_block;
       if (row >= job.N) return;
       const float al = (job.acc_out == nullptr) ? __ldg(job.alpha) : 0.f;
 #pragma unroll
-      for (int t = 0; t < T_PAD; ++t) {
-        if (t >= p.T) break;
-        const int a = v[t] - __ldg(job.codesum + t);
-        if (job.acc_out != nullptr) job.acc_out[(size_t)t * job.N + row] = a;
-        else job.y[(size_t)t * job.N + row] = __float2bfloat16_rn((float)a * (__ldg(job.scale + t) * al));
+      for (int t = 0; t < 16; ++t) {
+        const int tok = j * 16 + t;
+        if (tok >= p.T) break;
+        const int a = v[t] - __ldg(job.codesum + tok);
+        if (job.acc_out != nullptr) job.acc_out[(size_t)tok * job.N + row] = a;
+        else job.y[(size_t)tok * job.N + row] = __float2bfloat16_rn((float)a * (__ldg(job.scale + tok) * al));
       }
+    };
+    auto load_chunk = [&](int b, int j, int (&v)[16]) {
+      uint32_t r[16];
+      tmem_ld16(lane_base + (uint32_t)(b * D_COLS + j * 16), r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int t = 0; t < 16; ++t) v[t] = (int)r[t];
     };
     Range range(p, u0, u1);
     Segment sg;
     uint32_t seg = 0;
     bool ok = true;
-    int own[T_PAD];               // sums of the row block this CTA owns but does not complete (its last segment)
-    int own_rb = -1, own_job = 0;
+    // A row block this CTA owns but does not complete is its last segment: its sums stay in their
+    // D buffer until the other CTAs' parts have been added.
+    int own_b = -1, own_rb = 0, own_job = 0;
     long own_end = 0;
     while (range.next(sg)) {
       const int b = seg & 1;
       ok = ok && mbar_wait(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
-      int v[T_PAD];
+      ++seg;
+      const bool whole = sg.ka == 0 && sg.ke == p.jobs[sg.job].n_kb;
+      if (sg.ka == 0 && !whole) {
+        if (ok) { own_b = b; own_rb = sg.rb; own_job = sg.job; own_end = sg.rb_end; }
+        continue;
+      }
       if (ok) {
         tc_fence_after();
-#pragma unroll
+        const int n_chunks = (p.T + 15) / 16;
+#pragma unroll 1
         for (int j = 0; j < T_PAD / 16; ++j) {
-          uint32_t r[16];
-          tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * 64 + j * 16), r);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if (j >= n_chunks) break;                           // padded token columns are never read
+          int v[16];
+          load_chunk(b, j, v);
+          if (whole) {
+            finish_chunk(sg.job, sg.rb, j, v);
+          } else {
+            // not the owner: publish the partial sums ([token][128 rows], coalesced)
 #pragma unroll
-          for (int t = 0; t < 16; ++t) v[j * 16 + t] = (int)r[t];
+            for (int t = 0; t < 16; ++t) __stcg(p.part + ((size_t)c * T_PAD + j * 16 + t) * 128 + row_in_block, v[t]);
+          }
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&d_empty[b]);
       }
-      ++seg;
-      const bool whole = sg.ka == 0 && sg.ke == p.jobs[sg.job].n_kb;
-      if (sg.ka != 0) {
-        // not the owner: publish the partial sums ([t][128 rows], coalesced), then raise this CTA's flag
-        if (ok) {
-#pragma unroll
-          for (int t = 0; t < T_PAD; ++t) __stcg(p.part + ((size_t)c * T_PAD + t) * 128 + row_in_block, v[t]);
-          __threadfence();
-        }
-        named_barrier(3, 128);                                // all four epilogue warps have written
+      if (!whole) {
+        if (ok) __threadfence();
+        named_barrier(3, 128);                                // all four epilogue warps have written their rows
         if (ok && warp == 12 && lane == 0) atomicExch(p.flags + c, 1);
-      } else if (whole) {
-        if (ok) finish(sg.job, sg.rb, v);
-      } else if (ok) {
-#pragma unroll
-        for (int t = 0; t < T_PAD; ++t) own[t] = v[t];
-        own_rb = sg.rb;
-        own_job = sg.job;
-        own_end = sg.rb_end;
       }
     }
-    if (own_rb >= 0 && ok) {
+    if (own_b >= 0 && ok) {
       // the row block continues in the next CTAs: collect their parts (each was published before its CTA waits for anything)
-      const long end = own_end;
       int n_follow = 0;
-      while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < end) ++n_follow;
-      // wait for all of them at once: lane l polls the flags of followers l, l+32, ...
+      while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < own_end) ++n_follow;
       {
-        int ready = 1;
+        int ready = 1;                                        // lane l polls the flags of followers l, l+32, ...
         for (int f = lane; f < n_follow && ready; f += 32) {
           volatile int* flag = p.flags + c + 1 + f;
           const uint64_t t0 = global_ns();
@@ -386,34 +395,33 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
       }
       if (ok) {
         __threadfence();
-        // independent loads, four followers in flight at a time
-        for (int f0 = 0; f0 < n_follow; f0 += 4) {
-          int tmp[4][T_PAD <= 16 ? T_PAD : 1];
-          if constexpr (T_PAD <= 16) {
+        tc_fence_after();
+        const int n_chunks = (p.T + 15) / 16;
+#pragma unroll 1
+        for (int j = 0; j < T_PAD / 16; ++j) {
+          if (j >= n_chunks) break;
+          int v[16];
+          load_chunk(own_b, j, v);
+          for (int f0 = 0; f0 < n_follow; f0 += 4) {          // independent loads, four followers in flight
+            int tmp[4][16];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int f = f0 + j < n_follow ? f0 + j : n_follow - 1;
+            for (int q = 0; q < 4; ++q) {
+              const int f = f0 + q < n_follow ? f0 + q : n_follow - 1;
 #pragma unroll
-              for (int t = 0; t < T_PAD; ++t)
-                tmp[j][t] = __ldcg(p.part + ((size_t)(c + 1 + f) * T_PAD + t) * 128 + row_in_block);
+              for (int t = 0; t < 16; ++t)
+                tmp[q][t] = __ldcg(p.part + ((size_t)(c + 1 + f) * T_PAD + j * 16 + t) * 128 + row_in_block);
             }
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              if (f0 + j < n_follow) {
+            for (int q = 0; q < 4; ++q)
+              if (f0 + q < n_follow) {
 #pragma unroll
-                for (int t = 0; t < T_PAD; ++t) own[t] += tmp[j][t];
+                for (int t = 0; t < 16; ++t) v[t] += tmp[q][t];
               }
-          } else {
-            (void)tmp;
-            for (int j = 0; j < 4 && f0 + j < n_follow; ++j) {
-#pragma unroll
-              for (int t = 0; t < T_PAD; ++t)
-                own[t] += __ldcg(p.part + ((size_t)(c + 1 + f0 + j) * T_PAD + t) * 128 + row_in_block);
-            }
           }
+          finish_chunk(own_job, own_rb, j, v);
         }
+        tc_fence_before();
       }
-      if (ok) finish(own_job, own_rb, own);
     }
   }
 
@@ -461,7 +469,7 @@ int sm_count() {
   return n;
 }
 
-int pad_tokens(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
+int pad_tokens(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 128)); }
 
 template <int T_PAD, int KBP>
 int launch_variant(const CodeMaps& maps, const Params& p, int grid, cudaStream_t s) {
@@ -500,7 +508,7 @@ size_t gemm_stream_counter_words(int N) { (void)N; return MAX_GRID; }
 int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
                              int32_t* part, int* flags, cudaStream_t s) {
   if (T <= 0 || n_jobs <= 0) return HBL_OK;
-  if (T > 64) return HBL_ERR_TOO_LARGE;
+  if (T > 128) return HBL_ERR_TOO_LARGE;
   if (n_jobs > MAX_JOBS || n_inputs > MAX_MAPS || n_inputs <= 0) return HBL_ERR_SHAPE;
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return HBL_ERR_CUDA;
@@ -523,7 +531,7 @@ int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const Stre
   // Column blocks per unit: as wide as every K allows while every CTA still gets a few units.
   long blocks = 0;
   for (int j = 0; j < n_jobs; ++j) blocks += (long)((jobs[j].N + 127) / 128) * (inputs[jobs[j].input].K / 128);
-  int kbp = 4;
+  int kbp = t_pad > 64 ? 2 : 4;            // 128 token columns: the codes of a unit fill the stage, keep units at two blocks
   for (;;) {
     bool fits = blocks / kbp >= 4L * n_sm;
     for (int m = 0; m < n_inputs; ++m) fits = fits && (inputs[m].K / 128) % kbp == 0;
@@ -552,7 +560,8 @@ int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const Stre
   const int grid = (int)(u < n_sm ? u : n_sm);
   if (t_pad == 16) return launch_kbp<16>(kbp, maps, p, grid, s);
   if (t_pad == 32) return launch_kbp<32>(kbp, maps, p, grid, s);
-  return launch_kbp<64>(kbp, maps, p, grid, s);
+  if (t_pad == 64) return launch_kbp<64>(kbp, maps, p, grid, s);
+  return kbp == 2 ? launch_variant<128, 2>(maps, p, grid, s) : launch_variant<128, 1>(maps, p, grid, s);
 }
 
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
