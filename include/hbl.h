@@ -55,7 +55,7 @@ typedef enum { HBL_F32 = 0, HBL_BF16 = 1 } hbl_dtype_t;
 /* Which contraction kernel hbl_forward / hbl_gemm_i32 use. */
 typedef enum {
   HBL_PATH_AUTO = 0,       /* by token count */
-  HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers into tensor memory); tokens <= 128 */
+  HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers into tensor memory); tokens <= 512 */
   HBL_PATH_TENSOR = 2      /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
 } hbl_path_t;
 
@@ -168,7 +168,7 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
  * stream callback where an allocation would synchronise the device, a runtime
  * whose memory budget is frozen after initialisation -- and have no buffer of
  * their own to lend.  For them the kernel's scratch (partial sums handed between
- * thread blocks, and their ready flags) sits in a fixed 1.25 MiB + 1 KiB array inside
+ * thread blocks, and their ready flags) sits in a fixed 1.25 MiB + 4 KiB array inside
  * the library's device image; every GPU that loads the library holds it until the
  * process ends.
  *   - Inputs and the output are still the caller's: codes int8 [T,K], codesum

@@ -43,7 +43,7 @@ void profile_after(int kernel_id, cudaStream_t s) {
 
 namespace {
 
-constexpr int kStreamMaxTokens = 128;
+constexpr int kStreamMaxTokens = 512;     // = gemm_stream_max_tokens(): four passes of 128 token columns
 constexpr int kMaxInDim = 32768;
 
 struct ForwardWs {           // byte offsets inside the caller's workspace
@@ -83,8 +83,15 @@ int check_quant_args(int x_dtype, int in_dim, int bits, int use_hadamard, float 
   return HBL_OK;
 }
 
-int resolve_path(int path, int tokens) {
-  if (path == HBL_PATH_AUTO) return tokens <= kStreamMaxTokens ? HBL_PATH_STREAM : HBL_PATH_TENSOR;
+// Which contraction kernel.  The streaming kernel reads the packed weights once per 128 tokens: up to
+// 128 tokens it always wins; up to 512 it wins when there are enough weight bytes for its fixed costs
+// to disappear (measured: a 7B block yes, a single 2048 x 2048 layer no).
+int resolve_path(int path, int tokens, size_t packed_bytes) {
+  if (path == HBL_PATH_AUTO) {
+    if (tokens <= 128) return HBL_PATH_STREAM;
+    if (tokens <= kStreamMaxTokens && packed_bytes >= (size_t)16 << 20) return HBL_PATH_STREAM;
+    return HBL_PATH_TENSOR;
+  }
   if (path == HBL_PATH_STREAM) return tokens <= kStreamMaxTokens ? HBL_PATH_STREAM : -1;
   if (path == HBL_PATH_TENSOR) return HBL_PATH_TENSOR;
   return -2;
@@ -161,7 +168,7 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
   if (rc != HBL_OK) return rc;
   rc = check_quant_args(x_dtype, in_dim, bits, use_hadamard, eps);
   if (rc != HBL_OK) return rc;
-  const int p = resolve_path(path, tokens);
+  const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
   if (tokens == 0) return HBL_OK;
@@ -227,7 +234,7 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   rc = check_quant_args(b->x_dtype, H, b->bits, 1, b->eps);
   if (rc != HBL_OK) return rc;
   if (!is_pow2(F)) return HBL_ERR_NOT_POW2;
-  const int p = resolve_path(path, T);
+  const int p = resolve_path(path, T, ((size_t)4 * H * H + (size_t)3 * H * F) / 4);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
   if (T == 0) return HBL_OK;
@@ -353,7 +360,7 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
                  int out_dim, int32_t* acc_out, void* workspace, size_t workspace_bytes, int path, void* stream) {
   int rc = check_dims(tokens, in_dim, out_dim);
   if (rc != HBL_OK) return rc;
-  const int p = resolve_path(path, tokens);
+  const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
   if (tokens == 0) return HBL_OK;

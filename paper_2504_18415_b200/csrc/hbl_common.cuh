@@ -83,7 +83,8 @@ int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* c
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s);
 int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
                        const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s);
-// Several weight tensors, each reading one of up to four quantized inputs, in one launch (T <= 64).
+// Several weight tensors, each reading one of up to four quantized inputs, per launch; one launch per 128 tokens.
+int gemm_stream_max_tokens();
 struct StreamInput { const int8_t* codes; const float* scale; const int32_t* codesum; int K; };
 struct StreamJob { const void* W_packed; const float* alpha; __nv_bfloat16* y; int32_t* acc_out; int N; int input; };
 int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,

@@ -216,7 +216,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
           const int s = i % SW;
           unsigned char* st = stages + (size_t)s * STAGE_BYTES;
           if (i >= primed) {
-            if (!mbar_wait(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+            if (!mbar_wait<true>(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
             mbar_expect_tx(&w_full[s], STAGE_BYTES);
             bulk_load(st, job.Wp + ((size_t)sg.rb * job.n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[s]);
           }
@@ -274,8 +274,8 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
       for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
         if ((int)(i & 1) != group) continue;
         const int s = i % SW, a = i % NA;
-        ok = mbar_wait(&w_full[s], (i / SW) & 1, abort_flag, p.status) &&
-             mbar_wait(&a_empty[a], ((i / NA) & 1) ^ 1, abort_flag, p.status);
+        ok = mbar_wait<true>(&w_full[s], (i / SW) & 1, abort_flag, p.status) &&
+             mbar_wait<true>(&a_empty[a], ((i / NA) & 1) ^ 1, abort_flag, p.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -306,18 +306,32 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     const int quad = warp & 3;
     const int row_in_block = quad * 32 + lane;
     const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
-    auto finish_chunk = [&](int job_idx, int rb, int j, const int (&v)[16]) {
+    // The job's fields are copied to registers once per segment (the job table sits in parameter
+    // space; indexing it dynamically inside the store loop would re-read it every time).
+    struct Out { const float* scale; const int32_t* codesum; __nv_bfloat16* y; int32_t* acc_out; float al; int N; };
+    auto job_out = [&](int job_idx) {
       const Job& job = p.jobs[job_idx];
+      Out o;
+      o.scale = job.scale; o.codesum = job.codesum; o.y = job.y; o.acc_out = job.acc_out; o.N = job.N;
+      o.al = (job.acc_out == nullptr) ? __ldg(job.alpha) : 0.f;
+      return o;
+    };
+    auto finish_chunk = [&](const Out& o, int rb, int j, const int (&v)[16]) {
       const int row = rb * 128 + row_in_block;
-      if (row >= job.N) return;
-      const float al = (job.acc_out == nullptr) ? __ldg(job.alpha) : 0.f;
+      // lane t fetches token 16 j + t's code sum and scale; the values are handed round by shuffle
+      const int my_tok = j * 16 + (lane & 15);
+      const int my_cs = my_tok < p.T ? __ldg(o.codesum + my_tok) : 0;
+      const float my_f = (my_tok < p.T && o.acc_out == nullptr) ? __ldg(o.scale + my_tok) * o.al : 0.f;
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
         const int tok = j * 16 + t;
-        if (tok >= p.T) break;
-        const int a = v[t] - __ldg(job.codesum + tok);
-        if (job.acc_out != nullptr) job.acc_out[(size_t)tok * job.N + row] = a;
-        else job.y[(size_t)tok * job.N + row] = __float2bfloat16_rn((float)a * (__ldg(job.scale + tok) * al));
+        const int cs = __shfl_sync(0xffffffffu, my_cs, t);
+        const float f = __shfl_sync(0xffffffffu, my_f, t);
+        if (tok < p.T && row < o.N) {
+          const int a = v[t] - cs;
+          if (o.acc_out != nullptr) o.acc_out[(size_t)tok * o.N + row] = a;
+          else o.y[(size_t)tok * o.N + row] = __float2bfloat16_rn((float)a * f);
+        }
       }
     };
     auto load_chunk = [&](int b, int j, int (&v)[16]) {
@@ -337,7 +351,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     long own_end = 0;
     while (range.next(sg)) {
       const int b = seg & 1;
-      ok = ok && mbar_wait(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
+      ok = ok && mbar_wait<true>(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       ++seg;
       const bool whole = sg.ka == 0 && sg.ke == p.jobs[sg.job].n_kb;
@@ -347,6 +361,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
       }
       if (ok) {
         tc_fence_after();
+        const Out o = job_out(sg.job);
         const int n_chunks = (p.T + 15) / 16;
 #pragma unroll 1
         for (int j = 0; j < T_PAD / 16; ++j) {
@@ -354,7 +369,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
           int v[16];
           load_chunk(b, j, v);
           if (whole) {
-            finish_chunk(sg.job, sg.rb, j, v);
+            finish_chunk(o, sg.rb, j, v);
           } else {
             // not the owner: publish the partial sums ([token][128 rows], coalesced)
 #pragma unroll
@@ -396,6 +411,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
       if (ok) {
         __threadfence();
         tc_fence_after();
+        const Out o = job_out(own_job);
         const int n_chunks = (p.T + 15) / 16;
 #pragma unroll 1
         for (int j = 0; j < T_PAD / 16; ++j) {
@@ -418,7 +434,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
                 for (int t = 0; t < 16; ++t) v[t] += tmp[q][t];
               }
           }
-          finish_chunk(own_job, own_rb, j, v);
+          finish_chunk(o, own_rb, j, v);
         }
         tc_fence_before();
       }
@@ -500,12 +516,18 @@ int launch_kbp(int kbp, const CodeMaps& maps, const Params& p, int grid, cudaStr
 
 }  // namespace
 
-// Scratch of the streaming contraction: `part` slots (contents irrelevant on entry) and flags (zero on entry).
-size_t gemm_stream_acc_words(int T, int N) { (void)N; return (size_t)MAX_GRID * 128 * pad_tokens(T < 1 ? 1 : T); }
-size_t gemm_stream_counter_words(int N) { (void)N; return MAX_GRID; }
+// Scratch of the streaming contraction: `part` slots (contents irrelevant on entry) and flags (zero on
+// entry; one set per pass of 128 tokens).
+constexpr int kMaxPasses = 4;
+size_t gemm_stream_acc_words(int T, int N) {
+  (void)N;
+  return (size_t)MAX_GRID * 128 * pad_tokens(T < 1 ? 1 : (T > 128 ? 128 : T));
+}
+size_t gemm_stream_counter_words(int N) { (void)N; return (size_t)MAX_GRID * kMaxPasses; }
+int gemm_stream_max_tokens() { return 128 * kMaxPasses; }
 
-// Several weight tensors (each reading one of up to four quantized inputs) in one launch.
-int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
+// Several weight tensors (each reading one of up to four quantized inputs) in one launch, T <= 128.
+static int launch_gemm_stream_pass(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
                              int32_t* part, int* flags, cudaStream_t s) {
   if (T <= 0 || n_jobs <= 0) return HBL_OK;
   if (T > 128) return HBL_ERR_TOO_LARGE;
@@ -515,8 +537,9 @@ int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const Stre
   const int t_pad = pad_tokens(T);
   CodeMaps maps;
   for (int m = 0; m < MAX_MAPS; ++m) {
+    if (m >= n_inputs) { maps.m[m] = maps.m[0]; continue; }   // unused slots: any valid map
     // codes [T, K] int8 row-major; box = 128 bytes of K x t_pad tokens (rows beyond T read as zero), 128-byte swizzle
-    const StreamInput& in = inputs[m < n_inputs ? m : 0];
+    const StreamInput& in = inputs[m];
     cuuint64_t dims[2] = {(cuuint64_t)in.K, (cuuint64_t)T};
     cuuint64_t strides[1] = {(cuuint64_t)in.K};
     cuuint32_t box[2] = {128u, (cuuint32_t)t_pad};
@@ -557,11 +580,52 @@ int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const Stre
   p.status = device_status_word();
   if (p.status == nullptr) return HBL_ERR_CUDA;
   p.T = T;
-  const int grid = (int)(u < n_sm ? u : n_sm);
+  // Every CTA that shares a row block writes (and the owner reads) 128 x t_pad partial sums.  Use
+  // all SMs only when each one streams several times that in weights; otherwise fewer, fatter
+  // CTAs (never fewer than one per row block, which shares nothing).
+  long grid_l = u < n_sm ? u : n_sm;
+  {
+    long n_rb_all = 0, packed_bytes = 0;
+    for (int j = 0; j < n_jobs; ++j) {
+      n_rb_all += (jobs[j].N + 127) / 128;
+      packed_bytes += (long)((jobs[j].N + 127) / 128) * 128 * inputs[jobs[j].input].K / 4;
+    }
+    const long part_bytes = 128L * t_pad * 4;
+    long want = packed_bytes / (4 * part_bytes);
+    if (want < n_rb_all) want = n_rb_all;
+    if (want < grid_l) grid_l = want;
+    if (grid_l < 1) grid_l = 1;
+  }
+  const int grid = (int)grid_l;
   if (t_pad == 16) return launch_kbp<16>(kbp, maps, p, grid, s);
   if (t_pad == 32) return launch_kbp<32>(kbp, maps, p, grid, s);
   if (t_pad == 64) return launch_kbp<64>(kbp, maps, p, grid, s);
   return kbp == 2 ? launch_variant<128, 2>(maps, p, grid, s) : launch_variant<128, 1>(maps, p, grid, s);
+}
+
+// Up to 512 tokens: the weights stream once per 128 tokens (still far cheaper than expanding them to
+// int8 in HBM for the large-batch kernel, whose tiles would also be mostly padding at these sizes).
+int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
+                             int32_t* part, int* flags, cudaStream_t s) {
+  if (T <= 0 || n_jobs <= 0) return HBL_OK;
+  if (T > gemm_stream_max_tokens()) return HBL_ERR_TOO_LARGE;
+  if (n_jobs > MAX_JOBS || n_inputs > MAX_MAPS || n_inputs <= 0) return HBL_ERR_SHAPE;
+  for (int pass = 0; pass * 128 < T; ++pass) {
+    const int t0 = pass * 128, tn = T - t0 < 128 ? T - t0 : 128;
+    StreamInput in[MAX_MAPS];
+    StreamJob jb[MAX_JOBS];
+    for (int m = 0; m < n_inputs; ++m)
+      in[m] = {inputs[m].codes + (size_t)t0 * inputs[m].K, inputs[m].scale ? inputs[m].scale + t0 : nullptr,
+               inputs[m].codesum + t0, inputs[m].K};
+    for (int j = 0; j < n_jobs; ++j) {
+      jb[j] = jobs[j];
+      if (jb[j].y) jb[j].y += (size_t)t0 * jobs[j].N;
+      if (jb[j].acc_out) jb[j].acc_out += (size_t)t0 * jobs[j].N;
+    }
+    const int rc = launch_gemm_stream_pass(in, n_inputs, jb, n_jobs, tn, part, flags + pass * MAX_GRID, s);
+    if (rc != HBL_OK) return rc;
+  }
+  return HBL_OK;
 }
 
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,

@@ -10,7 +10,7 @@ using namespace hbl;
 namespace {
 
 constexpr size_t kStaticAccWords = 160 * 128 * 16;   // one 128-row x 16-token slot of partial sums per CTA (1.25 MiB): tokens <= 16
-constexpr size_t kStaticCounterWords = 256;          // one flag per CTA
+constexpr size_t kStaticCounterWords = 1024;         // the contraction's flag words (one per CTA and pass)
 constexpr size_t kStaticScratchBytes = (kStaticAccWords + kStaticCounterWords) * sizeof(int32_t);
 
 // Every GPU that loads the library holds this array until the process exits.

@@ -36,14 +36,30 @@ __device__ __forceinline__ uint64_t global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+// try_wait with a suspend-time hint: the hardware parks the thread until the phase completes or
+// the hint runs out, instead of having it re-issue the instruction back to back.
+__device__ __forceinline__ bool mbar_try_hint(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
 // Returns false when aborted (this thread's timeout, or another role's).
+// POLITE waiters (anything but the thread that feeds the tensor core) park between polls so that
+// they do not take issue slots from the warps that are on the critical path.
+template <bool POLITE = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
   if (mbar_try(bar, parity)) return true;
   if (*abort_flag) return false;
   const uint64_t t0 = global_ns();
   uint32_t polls = 0;
-  while (!mbar_try(bar, parity)) {
-    if ((++polls & 255u) == 0) {
+  for (;;) {
+    if (POLITE ? mbar_try_hint(bar, parity, 2000u) : mbar_try(bar, parity)) return true;
+    if (POLITE) __nanosleep(40);
+    if ((++polls & (POLITE ? 15u : 255u)) == 0) {
       if (*abort_flag) return false;
       if (global_ns() - t0 > 2000000000ull) {
         report_device_error(status, HBL_ERR_TIMEOUT);
@@ -52,7 +68,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
-  return true;
 }
 // Untiled bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completing on `bar`.
 __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {

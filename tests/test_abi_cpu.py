@@ -54,7 +54,7 @@ def test_argument_errors_come_before_any_launch(L):
     assert f(eps=float("nan")) == 7
     assert f(dt=7) == 10                       # HBL_ERR_FORMAT
     assert f(path=9) == 10
-    assert f(T=200, path=hbl.PATH_STREAM) == 11   # HBL_ERR_TOO_LARGE
+    assert f(T=600, path=hbl.PATH_STREAM) == 11   # HBL_ERR_TOO_LARGE
     assert f(K=65536) == 11
     assert f(T=0) == 0                         # no-op
     assert f(x=n) == 1                         # HBL_ERR_NULL

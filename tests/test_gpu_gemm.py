@@ -22,7 +22,7 @@ def setup(T, K, N, bits, seed):
 
 @pytest.mark.parametrize("T,K,N", [(1, 128, 16), (3, 384, 144), (8, 2048, 2048), (16, 8192, 2048),
                                    (17, 512, 528), (33, 4096, 1024), (64, 1024, 4096), (5, 16384, 256),
-                                   (100, 2048, 784), (128, 4096, 2048), (65, 384, 4112)])
+                                   (100, 2048, 784), (128, 4096, 2048), (65, 384, 4112), (300, 1024, 528), (512, 2048, 256)])
 @pytest.mark.parametrize("bits", [4, 8])
 def test_stream_kernel_bit_exact(T, K, N, bits):
     q, packed, wt = setup(T, K, N, bits, T * 1000 + K + N)
