@@ -137,6 +137,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// Tile order: groups of GROUP_M token blocks; inside a group the weight tiles are walked one column
+// of the group at a time.  The CTAs that run at the same time then share a few weight tiles and a
+// few token blocks (both stay in L2) instead of sweeping the whole weight matrix per token block.
+constexpr int GROUP_M = 8;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& m0, int& n0) {
+  const int per_group = GROUP_M * tiles_n;
+  const int first_m = (tile / per_group) * GROUP_M;
+  const int gm = tiles_m - first_m < GROUP_M ? tiles_m - first_m : GROUP_M;
+  const int local = tile % per_group;
+  m0 = (first_m + local % gm) * BM;
+  n0 = (local / gm) * BN;
+}
+
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const float* __restrict__ scale, const float* __restrict__ alpha,
@@ -179,7 +192,8 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        int m0, n0;
+        tile_coords(tile, tiles_m, tiles_n, m0, n0);
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abort_flag, status)) { ok = false; break; }
@@ -222,7 +236,8 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     uint32_t tl = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tl) {
       const int b = tl & 1;
-      const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+      int m0, n0;
+      tile_coords(tile, tiles_m, tiles_n, m0, n0);
       const bool got = mbar_wait(&tfull_bar[b], (tl >> 1) & 1, abort_flag, status);
       if (!__all_sync(0xffffffffu, got)) break;      // warp-uniform: tcgen05.ld needs the whole warp
       tc_fence_after();

@@ -112,6 +112,10 @@ unpack_kernel(const uint32_t* __restrict__ packed, int N, int K, int8_t* __restr
     o.w = __vsub4((wd >> 6) & 0x03030303u, 0x01010101u);
     *reinterpret_cast<uint4*>(out + (size_t)R * K + (size_t)kb * 128 + 16 * (4 * h + v)) = o;
   }
+  // Launched as a programmatic dependent of the activation kernel (it reads nothing of it, so the two
+  // overlap); completing only after that kernel keeps "unpack done" meaning "activations done" for
+  // the contraction that follows.
+  grid_dependency_wait();
 }
 
 }  // namespace
@@ -138,7 +142,7 @@ int launch_unpack_weights(const void* packed, int N, int K, int8_t* out, cudaStr
   const size_t n_words = (size_t)((N + 127) / 128) * (K / 128) * 1024;
   int grid = (int)min((size_t)148 * 16, (n_words + 255) / 256);
   profile_before(KERNEL_UNPACK, s);
-  unpack_kernel<<<grid, 256, 0, s>>>(static_cast<const uint32_t*>(packed), N, K, out);
+  HBL_CUDA_OK(launch_dependent(unpack_kernel, dim3(grid), dim3(256), 0, s, static_cast<const uint32_t*>(packed), N, K, out));
   profile_after(KERNEL_UNPACK, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
