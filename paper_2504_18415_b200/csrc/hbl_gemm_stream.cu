@@ -93,6 +93,12 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
+// One lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n .reg .pred p;\n elect.sync _|p, 0xffffffff;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -228,25 +234,30 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(T_PAD);
-      Range range(p, u0, u1);
-      Segment sg;
-      uint32_t i = 0, seg = 0;
-      bool ok = true;
-      while (ok && range.next(sg)) {
-        const int b = seg & 1;
-        if (!mbar_wait(&d_empty[b], ((seg >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+    // The whole warp walks the loop and one elected lane issues: in warp-uniform code the operands
+    // of tcgen05.mma (descriptors, tensor-memory addresses) live in uniform registers, and the
+    // instructions issue several times faster than from inside a single-lane branch.
+    const uint32_t idesc = make_idesc(T_PAD);
+    Range range(p, u0, u1);
+    Segment sg;
+    uint32_t i = 0, seg = 0;
+    bool ok = true;
+    while (ok && range.next(sg)) {
+      const int b = seg & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(&d_empty[b], ((seg >> 1) & 1) ^ 1, abort_flag, p.status));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(b * D_COLS);
+      for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
+        const int s = i % SW, a = i % NA;
+        // The unpack warps waited for the stage (weights and codes) before they filled the A buffer,
+        // so one wait covers both operands.
+        ok = __all_sync(0xffffffffu, mbar_wait(&a_full[a], (i / NA) & 1, abort_flag, p.status));
+        if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(b * D_COLS);
-        for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
-          const int s = i % SW, a = i % NA;
-          // The unpack warps waited for the stage (weights and codes) before they filled the A buffer,
-          // so one wait covers both operands.
-          if (!mbar_wait(&a_full[a], (i / NA) & 1, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t codes_sm = smem_u32(stages + (size_t)s * STAGE_BYTES + GEO::CODES_OFF);
-          const uint32_t a_tmem = tmem_base + A_COL0 + (uint32_t)(32 * KBP) * a;
+        const uint32_t codes_sm = smem_u32(stages + (size_t)s * STAGE_BYTES + GEO::CODES_OFF);
+        const uint32_t a_tmem = tmem_base + A_COL0 + (uint32_t)(32 * KBP) * a;
+        if (elect_one()) {
 #pragma unroll
           for (int j = 0; j < KBP; ++j) {
             const uint64_t bdesc = make_desc(codes_sm + j * (T_PAD * 128));
@@ -257,10 +268,11 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
           }
           umma_commit(&w_empty[s]);          // the stage's codes have been read
           umma_commit(&a_empty[a]);          // and so has the A buffer
+          if (kb == sg.ke - 1) umma_commit(&d_full[b]);   // same lane as the MMAs it tracks
         }
-        if (ok) umma_commit(&d_full[b]);
-        ++seg;
+        __syncwarp();
       }
+      ++seg;
     }
   } else if (warp >= 4 && warp < 12) {
     // ------------------------------ unpack ------------------------------
