@@ -11,11 +11,14 @@
 // shared memory either.  What crosses shared memory is the packed stream (once in
 // by bulk copy, once out by 128-bit loads) and the tokens' codes (TMA).
 //
-//   warp 0        producer: per 128-column block one bulk copy of a 4 KiB packed tile
-//                 and one TMA load of the codes [T_pad x 128], 16-stage ring
-//   warp 1        allocates tensor memory; one lane issues four MMAs per block
-//   warps 4..11   unpack: two groups of four warps (one per TMEM lane quadrant) take
-//                 alternate blocks into a ring of eight A buffers (32 columns each)
+//   warp 0        weight producer: one bulk copy per unit (KBP packed tiles of 4 KiB, contiguous),
+//                 the first ring-full issued before anything else in the kernel
+//   warp 2        codes producer: TMA loads of the unit's codes [T_pad x 128] per column block,
+//                 a ring of their own
+//   warp 1 (, 3)  warp 1 allocates tensor memory; an issuer warp stays converged and one elected
+//                 lane issues the MMAs; up to 32 token columns warps 1 and 3 issue half a unit each
+//   warps 4..11   unpack: two groups of four warps (one per TMEM lane quadrant) take alternate
+//                 units and hand the weight stage back as soon as its words are in registers
 //   warps 12..15  epilogue: read the accumulators (two D buffers alternate), subtract
 //                 the code sum (weights are fed as u = w + 1), rescale, store bf16
 //
@@ -36,13 +39,17 @@ namespace {
 using namespace pipe;
 
 constexpr int THREADS = 512;
-constexpr int MAX_SW = 12;             // shared-memory stages (packed tiles + codes of one unit)
+constexpr int MAX_SW = 16;             // weight stages in shared memory
+constexpr int MAX_SC = 8;              // codes stages
 constexpr int MAX_NA = 12;             // A buffers in tensor memory
 // Tensor memory: two D buffers of D_COLS columns each, then the A buffers.
 constexpr int SMEM_RING_BYTES = 192 * 1024;
 constexpr int TMEM_COLS = 512;
 constexpr int TILE_BYTES = 4096;       // 128 rows x 128 columns x 2 bits
 constexpr int MAX_GRID = 160;
+// The unpack warps leave each 2-bit field u = w + 1 in the top two bits of its byte (a left shift
+// and a mask; no right shifts), so the MMA sees 64 u and every accumulator is an exact multiple of 64.
+constexpr int WEIGHT_SHIFT = 6;
 
 constexpr int MAX_JOBS = 8;            // weight tensors contracted by one launch (a decoder block has seven)
 constexpr int MAX_MAPS = 4;            // distinct quantized inputs they read (a decoder block has four)
@@ -99,17 +106,28 @@ __device__ __forceinline__ bool elect_one() {
   asm volatile("{\n .reg .pred p;\n elect.sync _|p, 0xffffffff;\n selp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
   return pred != 0;
 }
+// A whole warp waits on a barrier and stays converged.  (Measured: a wait that is satisfied at once
+// costs the warp about 95 cycles this way, about 150 when one lane polls and hands the outcome
+// round, and the whole kernel ran slower with single-lane polling -- so every lane polls, and the
+// serial loops below are arranged to need as few waits per unit as possible.)
+template <bool POLITE>
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  return __all_sync(0xffffffffu, mbar_wait<POLITE>(bar, parity, abort_flag, status));
+}
+template <bool POLITE>
+__device__ __forceinline__ bool warp_wait2(uint64_t* bar0, uint32_t parity0, uint64_t* bar1, uint32_t parity1,
+                                           volatile int* abort_flag, int* status) {
+  return __all_sync(0xffffffffu, mbar_wait<POLITE>(bar0, parity0, abort_flag, status) &&
+                                     mbar_wait<POLITE>(bar1, parity1, abort_flag, status));
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
       ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -143,43 +161,81 @@ struct Range {
   }
 };
 
-// A unit of work is KBP consecutive 128-column blocks of one row block: the single MMA-issuing
-// thread pays one barrier wait and two commits per unit, so wider units keep it ahead of the stream.
+// A unit of work is KBP consecutive 128-column blocks of one row block.  Its packed weights are one
+// contiguous run of KBP x 4 KiB (one bulk copy: copies of 16 KiB or more are what keeps HBM busy),
+// its codes KBP boxes of [T_PAD x 128].  The two travel in rings of their own: a weight stage is
+// handed back as soon as the unpack warps hold its words in registers, a codes stage when the MMAs
+// that read it have completed.
 template <int T_PAD, int KBP>
 struct Geo {
-  static constexpr int STAGE_BYTES = KBP * (TILE_BYTES + T_PAD * 128);
-  static constexpr int SW_RAW = SMEM_RING_BYTES / STAGE_BYTES;
-  static constexpr int SW = SW_RAW > MAX_SW ? MAX_SW : SW_RAW;
-  static constexpr int D_COLS = T_PAD < 64 ? 64 : T_PAD;          // columns of one accumulator buffer
+  static constexpr int W_BYTES = KBP * TILE_BYTES;
+  static constexpr int C_BYTES = KBP * T_PAD * 128;
+  // The codes come from L2 but queue behind the weight traffic, so they need the same lookahead
+  // in units as the weights: the ring bytes are split into equally many stages of each.
+  static constexpr int SC_RAW = SMEM_RING_BYTES / (C_BYTES + W_BYTES);
+  static constexpr int SC_CAP = SC_RAW > MAX_SC ? MAX_SC : SC_RAW;
+  static constexpr int SC = SC_CAP > 1 ? (SC_CAP & ~1) : SC_CAP;   // even: a stage stays with one issuer
+  static constexpr int SW_RAW = (SMEM_RING_BYTES - SC * C_BYTES) / W_BYTES;
+  static constexpr int SW_CAP = SW_RAW > MAX_SW ? MAX_SW : SW_RAW;
+  static constexpr int SW = SW_CAP & ~1;                          // even: a stage stays with one unpack group
+  // One thread issues an MMA every ~25 cycles, a unit of four tiles takes sixteen plus the waits and
+  // commits around them: more than the ~700 cycles in which HBM delivers the unit.  Up to 32 token
+  // columns two warps issue, each one half of every unit's MMAs into an accumulator of its own (the
+  // epilogue adds the two).  Both walk the units in the same order, so every barrier still sees its
+  // phases complete one at a time (issuers on alternate units would let one run two phases ahead of
+  // the other, which a parity wait cannot tell from "not yet").  Beyond 32 columns tensor memory has
+  // no room for the second accumulator set and the path is no longer bound by the weight stream.
+  static constexpr int ISSUERS = T_PAD <= 32 ? 2 : 1;
+  static constexpr int D_COLS = T_PAD < 64 ? 64 : T_PAD;          // columns of one accumulator buffer (all issuers)
+  static constexpr int D_ISSUER_COLS = D_COLS / ISSUERS;
   static constexpr int A_COL0 = 2 * D_COLS;
   static constexpr int NA_RAW = (TMEM_COLS - A_COL0) / (32 * KBP);
   static constexpr int NA = NA_RAW > MAX_NA ? MAX_NA : NA_RAW;
-  static constexpr int CODES_OFF = KBP * TILE_BYTES;
+  static constexpr int W_OFF = SC * C_BYTES;                      // codes ring first (1024-byte aligned boxes)
+  static constexpr size_t SMEM = (size_t)SC * C_BYTES + (size_t)SW * W_BYTES + 1024;
 };
 
 template <int T_PAD, int KBP>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant__ Params p) {
   using GEO = Geo<T_PAD, KBP>;
-  constexpr int STAGE_BYTES = GEO::STAGE_BYTES, SW = GEO::SW, NA = GEO::NA, D_COLS = GEO::D_COLS, A_COL0 = GEO::A_COL0;
+  constexpr int SW = GEO::SW, SC = GEO::SC, NA = GEO::NA, D_COLS = GEO::D_COLS, A_COL0 = GEO::A_COL0;
+  constexpr int W_BYTES = GEO::W_BYTES, C_BYTES = GEO::C_BYTES, ISSUERS = GEO::ISSUERS;
   extern __shared__ unsigned char smem_dyn[];
-  __shared__ __align__(8) uint64_t w_full[MAX_SW], w_empty[MAX_SW], a_full[MAX_NA], a_empty[MAX_NA], d_full[2], d_empty[2];
+  __shared__ __align__(8) uint64_t w_full[MAX_SW], w_empty[MAX_SW], c_full[MAX_SC], c_empty[MAX_SC], a_full[MAX_NA],
+      a_empty[MAX_NA], d_full[2], d_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
-  unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  unsigned char* c_ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  unsigned char* w_ring = c_ring + GEO::W_OFF;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long U = p.U;
   const int G = gridDim.x, c = blockIdx.x;
   const long u0 = U * c / G, u1 = U * (c + 1) / G;
 
+  uint32_t primed = 0;
   if (tid == 0) {
-    for (int s = 0; s < SW; ++s) { mbar_init(&w_full[s], 1); mbar_init(&w_empty[s], 1); }
-    for (int a = 0; a < NA; ++a) { mbar_init(&a_full[a], 4); mbar_init(&a_empty[a], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&d_full[b], 1); mbar_init(&d_empty[b], 4); }
+    for (int s = 0; s < SW; ++s) { mbar_init(&w_full[s], 1); mbar_init(&w_empty[s], 4); }
+    for (int s = 0; s < SC; ++s) { mbar_init(&c_full[s], 1); mbar_init(&c_empty[s], ISSUERS); }
+    for (int a = 0; a < NA; ++a) { mbar_init(&a_full[a], 4); mbar_init(&a_empty[a], ISSUERS); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&d_full[b], ISSUERS); mbar_init(&d_empty[b], 4); }
     abort_flag_s = 0;
     mbar_fence_init();
+    // The packed weights depend on no earlier kernel: the first ring-full of copies leaves before
+    // the CTA has even allocated its tensor memory, and (programmatic dependent launch) while the
+    // kernel that quantizes the activations may still be running.
+    Range range(p, u0, u1);
+    Segment sg;
+    while (primed < (uint32_t)SW && range.next(sg)) {
+      const Job& job = p.jobs[sg.job];
+      for (int kb = sg.ka; kb < sg.ke && primed < (uint32_t)SW; ++kb, ++primed) {
+        mbar_expect_tx(&w_full[primed], W_BYTES);
+        bulk_load(w_ring + (size_t)primed * W_BYTES, job.Wp + ((size_t)sg.rb * job.n_kb + kb) * W_BYTES, W_BYTES,
+                  &w_full[primed]);
+      }
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
@@ -192,51 +248,50 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
   const uint32_t tmem_base = tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------ producer ------------------------------
+    // ------------------------------ weight producer ------------------------------
     if (lane == 0) {
-      // The packed weights do not depend on the kernel that quantizes the activations: when this
-      // kernel was launched early (programmatic dependent launch) the first ring-full of weight
-      // copies is in flight before that kernel has finished.  The codes are fetched after the wait.
-      uint32_t primed = 0;
-      {
-        Range range(p, u0, u1);
-        Segment sg;
-        while (primed < (uint32_t)SW && range.next(sg)) {
-          const Job& job = p.jobs[sg.job];
-          for (int kb = sg.ka; kb < sg.ke && primed < (uint32_t)SW; ++kb, ++primed) {
-            mbar_expect_tx(&w_full[primed], STAGE_BYTES);
-            bulk_load(stages + (size_t)primed * STAGE_BYTES,
-                      job.Wp + ((size_t)sg.rb * job.n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[primed]);
-          }
-        }
-      }
-      grid_dependency_wait();
       Range range(p, u0, u1);
       Segment sg;
       uint32_t i = 0;
       bool ok = true;
       while (ok && range.next(sg)) {
         const Job& job = p.jobs[sg.job];
-        const CUtensorMap* tm_codes = &maps.m[job.map];
         for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
+          if (i < primed) continue;
           const int s = i % SW;
-          unsigned char* st = stages + (size_t)s * STAGE_BYTES;
-          if (i >= primed) {
-            if (!mbar_wait<true>(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
-            mbar_expect_tx(&w_full[s], STAGE_BYTES);
-            bulk_load(st, job.Wp + ((size_t)sg.rb * job.n_kb + kb) * (KBP * TILE_BYTES), KBP * TILE_BYTES, &w_full[s]);
-          }
-#pragma unroll
-          for (int j = 0; j < KBP; ++j)
-            tma_load_2d(st + GEO::CODES_OFF + j * (T_PAD * 128), tm_codes, &w_full[s], (kb * KBP + j) * 128, 0);
+          if (!mbar_wait<true>(&w_empty[s], ((i / SW) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+          mbar_expect_tx(&w_full[s], W_BYTES);
+          bulk_load(w_ring + (size_t)s * W_BYTES, job.Wp + ((size_t)sg.rb * job.n_kb + kb) * W_BYTES, W_BYTES, &w_full[s]);
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+  } else if (warp == 2) {
+    // ------------------------------ codes producer ------------------------------
+    if (lane == 0) {
+      grid_dependency_wait();                                  // the codes come from the previous kernel
+      Range range(p, u0, u1);
+      Segment sg;
+      uint32_t i = 0;
+      bool ok = true;
+      while (ok && range.next(sg)) {
+        const CUtensorMap* tm_codes = &maps.m[p.jobs[sg.job].map];
+        for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
+          const int s = i % SC;
+          if (i >= (uint32_t)SC && !mbar_wait<true>(&c_empty[s], ((i / SC) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+          mbar_expect_tx(&c_full[s], C_BYTES);
+#pragma unroll
+          for (int j = 0; j < KBP; ++j)
+            tma_load_2d(c_ring + (size_t)s * C_BYTES + j * (T_PAD * 128), tm_codes, &c_full[s], (kb * KBP + j) * 128, 0);
+        }
+      }
+    }
+  } else if (warp == 1 || (ISSUERS == 2 && warp == 3)) {
+    // ------------------------------ MMA issuer(s) ------------------------------
     // The whole warp walks the loop and one elected lane issues: in warp-uniform code the operands
     // of tcgen05.mma (descriptors, tensor-memory addresses) live in uniform registers, and the
     // instructions issue several times faster than from inside a single-lane branch.
+    const int g = warp >> 1;                                   // issuer 0 or 1
+    constexpr int MMAS = 4 * KBP / ISSUERS;                    // this issuer's share of a unit's MMAs
     const uint32_t idesc = make_idesc(T_PAD);
     Range range(p, u0, u1);
     Segment sg;
@@ -244,38 +299,44 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     bool ok = true;
     while (ok && range.next(sg)) {
       const int b = seg & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(&d_empty[b], ((seg >> 1) & 1) ^ 1, abort_flag, p.status));
+      ok = warp_wait<false>(&d_empty[b], ((seg >> 1) & 1) ^ 1, abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t d_tmem = tmem_base + (uint32_t)(b * D_COLS);
+      const uint32_t d_tmem = tmem_base + (uint32_t)(b * D_COLS + g * GEO::D_ISSUER_COLS);
+      uint32_t accumulate = 0;                                 // this issuer's first MMA of the segment overwrites
       for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
-        const int s = i % SW, a = i % NA;
-        // The unpack warps waited for the stage (weights and codes) before they filled the A buffer,
-        // so one wait covers both operands.
-        ok = __all_sync(0xffffffffu, mbar_wait(&a_full[a], (i / NA) & 1, abort_flag, p.status));
+        const int s = i % SC, a = i % NA;
+        // The unpack warps waited for the unit's codes before they filled the A buffer, so this one
+        // wait covers both operands.
+        ok = warp_wait<false>(&a_full[a], (i / NA) & 1, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t codes_sm = smem_u32(stages + (size_t)s * STAGE_BYTES + GEO::CODES_OFF);
+        const uint32_t codes_sm = smem_u32(c_ring + (size_t)s * C_BYTES);
         const uint32_t a_tmem = tmem_base + A_COL0 + (uint32_t)(32 * KBP) * a;
         if (elect_one()) {
 #pragma unroll
-          for (int j = 0; j < KBP; ++j) {
+          for (int q = 0; q < MMAS; ++q) {
+            const int m = g * MMAS + q, j = m >> 2, ks = m & 3;   // MMA m of the unit: tile j, K step ks
             const uint64_t bdesc = make_desc(codes_sm + j * (T_PAD * 128));
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              umma_i8_tmem_a(d_tmem, a_tmem + 32u * j + 8u * ks, bdesc + (uint64_t)(2 * ks), idesc,
-                             (kb > sg.ka) || j > 0 || ks > 0);
+            umma_i8_tmem_a(d_tmem, a_tmem + 32u * j + 8u * ks, bdesc + (uint64_t)(2 * ks), idesc,
+                           accumulate | (uint32_t)(q > 0));
           }
-          umma_commit(&w_empty[s]);          // the stage's codes have been read
+          umma_commit(&c_empty[s]);          // the stage's codes have been read
           umma_commit(&a_empty[a]);          // and so has the A buffer
-          if (kb == sg.ke - 1) umma_commit(&d_full[b]);   // same lane as the MMAs it tracks
         }
+        accumulate = 1;
         __syncwarp();
       }
+      // elect.sync names the same lane for the same mask every time, so this commit tracks the MMAs above
+      if (ok && elect_one()) umma_commit(&d_full[b]);
+      __syncwarp();
       ++seg;
     }
   } else if (warp >= 4 && warp < 12) {
     // ------------------------------ unpack ------------------------------
+    // Two groups of four warps (one per TMEM lane quadrant) take alternate units, so one group's
+    // waits and tensor-memory stores overlap the other's arithmetic.  A warp first pulls all of the
+    // unit's words for its 32 rows into registers, then expands them tile by tile.
     const int group = (warp - 4) >> 2, quad = warp & 3;
     const int row = quad * 32 + lane;
     Range range(p, u0, u1);
@@ -285,25 +346,36 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     while (ok && range.next(sg)) {
       for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
         if ((int)(i & 1) != group) continue;
-        const int s = i % SW, a = i % NA;
-        ok = mbar_wait<true>(&w_full[s], (i / SW) & 1, abort_flag, p.status) &&
-             mbar_wait<true>(&a_empty[a], ((i / NA) & 1) ^ 1, abort_flag, p.status);
-        ok = __all_sync(0xffffffffu, ok);
+        const int s = i % SW, sc = i % SC, a = i % NA;
+        ok = warp_wait<true>(&w_full[s], (i / SW) & 1, abort_flag, p.status);
         if (!ok) break;
-        tc_fence_after();
-        const unsigned char* st = stages + (size_t)s * STAGE_BYTES;
+        const unsigned char* st = w_ring + (size_t)s * W_BYTES + row * 16;
+        uint4 w4[KBP][2];
 #pragma unroll
         for (int j = 0; j < KBP; ++j) {
-          const uint4 lo = *reinterpret_cast<const uint4*>(st + j * TILE_BYTES + row * 16);
-          const uint4 hi = *reinterpret_cast<const uint4*>(st + j * TILE_BYTES + 2048 + row * 16);
-          const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-          uint32_t r[32];
-#pragma unroll
-          for (int kq = 0; kq < 8; ++kq)
-#pragma unroll
-            for (int q = 0; q < 4; ++q) r[kq * 4 + q] = (w[kq] >> (2 * q)) & 0x03030303u;   // column kq*4+q: k = 16 kq + 4 q + byte
-          tmem_st32(tmem_base + A_COL0 + (uint32_t)(32 * KBP) * a + 32u * j + ((uint32_t)(quad * 32) << 16), r);
+          w4[j][0] = *reinterpret_cast<const uint4*>(st + j * TILE_BYTES);
+          w4[j][1] = *reinterpret_cast<const uint4*>(st + j * TILE_BYTES + 2048);
         }
+        // the codes must have landed before the MMA warp is told that the unit is ready
+        ok = warp_wait2<true>(&c_full[sc], (i / SC) & 1, &a_empty[a], ((i / NA) & 1) ^ 1, abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = tmem_base + A_COL0 + (uint32_t)(32 * KBP) * a + ((uint32_t)(quad * 32) << 16);
+#pragma unroll
+        for (int j = 0; j < KBP; ++j) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const uint32_t w[4] = {w4[j][h].x, w4[j][h].y, w4[j][h].z, w4[j][h].w};
+            uint32_t r[16];
+#pragma unroll
+            for (int kq = 0; kq < 4; ++kq)
+#pragma unroll
+              for (int q = 0; q < 4; ++q) r[kq * 4 + q] = (w[kq] << (6 - 2 * q)) & 0xC0C0C0C0u;   // k = 64 h + 16 kq + 4 q + byte
+            tmem_st16(a_addr + 32u * j + 16u * h, r);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&w_empty[s]);               // the words are in registers: the stage can be refilled
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         tc_fence_before();
         __syncwarp();
@@ -328,19 +400,26 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
       o.al = (job.acc_out == nullptr) ? __ldg(job.alpha) : 0.f;
       return o;
     };
-    auto finish_chunk = [&](const Out& o, int rb, int j, const int (&v)[16]) {
-      const int row = rb * 128 + row_in_block;
-      // lane t fetches token 16 j + t's code sum and scale; the values are handed round by shuffle
+    // Lane t (mod 16) fetches the code sum and the scale of token 16 j + t; finish_chunk hands them
+    // round by shuffle.  Fetched ahead of the wait for the accumulators, so the loads overlap it.
+    struct Tok { int cs; float s; };
+    auto fetch_tok = [&](const Out& o, int j) {
       const int my_tok = j * 16 + (lane & 15);
-      const int my_cs = my_tok < p.T ? __ldg(o.codesum + my_tok) : 0;
-      const float my_f = (my_tok < p.T && o.acc_out == nullptr) ? __ldg(o.scale + my_tok) * o.al : 0.f;
+      Tok t;
+      t.cs = my_tok < p.T ? __ldg(o.codesum + my_tok) : 0;
+      t.s = (my_tok < p.T && o.acc_out == nullptr) ? __ldg(o.scale + my_tok) : 0.f;
+      return t;
+    };
+    auto finish_chunk = [&](const Out& o, int rb, int j, const Tok& mine, const int (&v)[16]) {
+      const int row = rb * 128 + row_in_block;
+      const float my_f = mine.s * o.al;
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
         const int tok = j * 16 + t;
-        const int cs = __shfl_sync(0xffffffffu, my_cs, t);
+        const int cs = __shfl_sync(0xffffffffu, mine.cs, t);
         const float f = __shfl_sync(0xffffffffu, my_f, t);
         if (tok < p.T && row < o.N) {
-          const int a = v[t] - cs;
+          const int a = (v[t] >> WEIGHT_SHIFT) - cs;
           if (o.acc_out != nullptr) o.acc_out[(size_t)tok * o.N + row] = a;
           else o.y[(size_t)tok * o.N + row] = __float2bfloat16_rn((float)a * f);
         }
@@ -352,7 +431,14 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
       for (int t = 0; t < 16; ++t) v[t] = (int)r[t];
+      if (ISSUERS == 2) {
+        tmem_ld16(lane_base + (uint32_t)(b * D_COLS + GEO::D_ISSUER_COLS + j * 16), r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int t = 0; t < 16; ++t) v[t] += (int)r[t];
+      }
     };
+    const int n_chunks = (p.T + 15) / 16;
     Range range(p, u0, u1);
     Segment sg;
     uint32_t seg = 0;
@@ -363,25 +449,26 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     long own_end = 0;
     while (range.next(sg)) {
       const int b = seg & 1;
-      ok = ok && mbar_wait<true>(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
-      ok = __all_sync(0xffffffffu, ok);
-      ++seg;
       const bool whole = sg.ka == 0 && sg.ke == p.jobs[sg.job].n_kb;
-      if (sg.ka == 0 && !whole) {
+      const bool own_partial = sg.ka == 0 && !whole;
+      Out o;
+      Tok tok0 = {0, 0.f};
+      if (whole) { o = job_out(sg.job); tok0 = fetch_tok(o, 0); }
+      ok = ok && warp_wait<true>(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
+      ++seg;
+      if (own_partial) {
         if (ok) { own_b = b; own_rb = sg.rb; own_job = sg.job; own_end = sg.rb_end; }
         continue;
       }
       if (ok) {
         tc_fence_after();
-        const Out o = job_out(sg.job);
-        const int n_chunks = (p.T + 15) / 16;
 #pragma unroll 1
         for (int j = 0; j < T_PAD / 16; ++j) {
           if (j >= n_chunks) break;                           // padded token columns are never read
           int v[16];
           load_chunk(b, j, v);
           if (whole) {
-            finish_chunk(o, sg.rb, j, v);
+            finish_chunk(o, sg.rb, j, j == 0 ? tok0 : fetch_tok(o, j), v);
           } else {
             // not the owner: publish the partial sums ([token][128 rows], coalesced)
 #pragma unroll
@@ -400,6 +487,8 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     }
     if (own_b >= 0 && ok) {
       // the row block continues in the next CTAs: collect their parts (each was published before its CTA waits for anything)
+      const Out o = job_out(own_job);
+      const Tok tok0 = fetch_tok(o, 0);
       int n_follow = 0;
       while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < own_end) ++n_follow;
       {
@@ -423,8 +512,6 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
       if (ok) {
         __threadfence();
         tc_fence_after();
-        const Out o = job_out(own_job);
-        const int n_chunks = (p.T + 15) / 16;
 #pragma unroll 1
         for (int j = 0; j < T_PAD / 16; ++j) {
           if (j >= n_chunks) break;
@@ -446,7 +533,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
                 for (int t = 0; t < 16; ++t) v[t] += tmp[q][t];
               }
           }
-          finish_chunk(o, own_rb, j, v);
+          finish_chunk(o, own_rb, j, j == 0 ? tok0 : fetch_tok(o, j), v);
         }
         tc_fence_before();
       }
@@ -502,7 +589,7 @@ int pad_tokens(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 12
 template <int T_PAD, int KBP>
 int launch_variant(const CodeMaps& maps, const Params& p, int grid, cudaStream_t s) {
   using GEO = Geo<T_PAD, KBP>;
-  constexpr size_t smem = (size_t)GEO::SW * GEO::STAGE_BYTES + 1024;
+  constexpr size_t smem = GEO::SMEM;
   auto kern = gemm_stream_kernel<T_PAD, KBP>;
   static bool done = false;   // idempotent attribute; a race only repeats the call
   if (!done) {
