@@ -96,6 +96,12 @@ __device__ __forceinline__ void umma_i8_tmem_a(uint32_t d_tmem, uint32_t a_tmem,
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Acquire load at GPU scope: what the writer stored before its release of the flag is visible after it.
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
@@ -445,19 +451,26 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     bool ok = true;
     // A row block this CTA owns but does not complete is its last segment: its sums stay in their
     // D buffer until the other CTAs' parts have been added.
-    int own_b = -1, own_rb = 0, own_job = 0;
-    long own_end = 0;
+    int own_b = -1, own_rb = 0, n_follow = 0;
+    Out own_o = {};
+    Tok own_tok0 = {0, 0.f};
     while (range.next(sg)) {
       const int b = seg & 1;
       const bool whole = sg.ka == 0 && sg.ke == p.jobs[sg.job].n_kb;
       const bool own_partial = sg.ka == 0 && !whole;
       Out o;
       Tok tok0 = {0, 0.f};
-      if (whole) { o = job_out(sg.job); tok0 = fetch_tok(o, 0); }
+      if (whole || own_partial) { o = job_out(sg.job); tok0 = fetch_tok(o, 0); }
+      if (own_partial) {
+        // Everything that needs neither the accumulators nor the other CTAs' parts happens before the
+        // wait: this segment is the CTA's last, so what follows it is the tail of the whole kernel.
+        own_o = o; own_tok0 = tok0;
+        while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < sg.rb_end) ++n_follow;
+      }
       ok = ok && warp_wait<true>(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
       ++seg;
       if (own_partial) {
-        if (ok) { own_b = b; own_rb = sg.rb; own_job = sg.job; own_end = sg.rb_end; }
+        if (ok) { own_b = b; own_rb = sg.rb; }
         continue;
       }
       if (ok) {
@@ -487,16 +500,15 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     }
     if (own_b >= 0 && ok) {
       // the row block continues in the next CTAs: collect their parts (each was published before its CTA waits for anything)
-      const Out o = job_out(own_job);
-      const Tok tok0 = fetch_tok(o, 0);
-      int n_follow = 0;
-      while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < own_end) ++n_follow;
+      const Out& o = own_o;
+      const Tok& tok0 = own_tok0;
       {
         int ready = 1;                                        // lane l polls the flags of followers l, l+32, ...
         for (int f = lane; f < n_follow && ready; f += 32) {
-          volatile int* flag = p.flags + c + 1 + f;
+          const int* flag = p.flags + c + 1 + f;
+          if (ld_acquire(flag)) continue;                     // the usual case: published long ago
           const uint64_t t0 = global_ns();
-          while (!*flag) {
+          while (!ld_acquire(flag)) {
             if (*abort_flag) { ready = 0; break; }
             if (global_ns() - t0 > 2000000000ull) {
               report_device_error(p.status, HBL_ERR_TIMEOUT);
@@ -510,7 +522,6 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
         ok = __all_sync(0xffffffffu, ready);
       }
       if (ok) {
-        __threadfence();
         tc_fence_after();
 #pragma unroll 1
         for (int j = 0; j < T_PAD / 16; ++j) {
