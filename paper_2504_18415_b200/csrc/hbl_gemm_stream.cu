@@ -60,12 +60,12 @@ struct Job {
   const unsigned char* Wp; const float* scale; const int32_t* codesum; const float* alpha;
   __nv_bfloat16* y; int32_t* acc_out;
   int N, n_kb, map;
-  long u_begin;
+  uint32_t u_begin;
 };
 struct Params {
   Job jobs[MAX_JOBS];
   int n_jobs;
-  long U;             // units of all jobs
+  uint32_t U;         // units of all jobs (U * grid fits 32 bits: checked on the host)
   int32_t* part;      // [grid][t_pad][128] partial sums of row blocks this CTA does not own
   int* flags;         // [grid], zero on entry
   int* status;
@@ -146,21 +146,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 
 // One contiguous piece of a CTA's range: units [ka, ke) of row block rb of one job.
-struct Segment { int job, rb, ka, ke; long rb_end; /* global index one past the row block's last unit */ };
+struct Segment { int job, rb, ka, ke; uint32_t rb_end; /* global index one past the row block's last unit */ };
 struct Range {
   const Params& p;
-  long u1, pos;
-  __device__ Range(const Params& p_, long u0_, long u1_) : p(p_), u1(u1_), pos(u0_) {}
+  uint32_t u1, pos;   // 32-bit on purpose: every role walks its range with these divisions
+  __device__ Range(const Params& p_, uint32_t u0_, uint32_t u1_) : p(p_), u1(u1_), pos(u0_) {}
   __device__ bool next(Segment& s) {
     if (pos >= u1) return false;
     int j = 0;
     while (j + 1 < p.n_jobs && pos >= p.jobs[j + 1].u_begin) ++j;
-    const long local = pos - p.jobs[j].u_begin;
-    const int n_kb = p.jobs[j].n_kb;
+    const uint32_t local = pos - p.jobs[j].u_begin;
+    const uint32_t n_kb = (uint32_t)p.jobs[j].n_kb;
     s.job = j;
     s.rb = (int)(local / n_kb);
     s.ka = (int)(local % n_kb);
-    s.rb_end = p.jobs[j].u_begin + (long)(s.rb + 1) * n_kb;
+    s.rb_end = p.jobs[j].u_begin + (uint32_t)(s.rb + 1) * n_kb;
     s.ke = (int)((u1 < s.rb_end ? u1 : s.rb_end) - (s.rb_end - n_kb));
     pos = s.rb_end - n_kb + s.ke;
     return true;
@@ -217,11 +217,10 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
   unsigned char* w_ring = c_ring + GEO::W_OFF;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const long U = p.U;
+  const uint32_t U = p.U;
   const int G = gridDim.x, c = blockIdx.x;
-  const long u0 = U * c / G, u1 = U * (c + 1) / G;
+  const uint32_t u0 = U * (uint32_t)c / (uint32_t)G, u1 = U * (uint32_t)(c + 1) / (uint32_t)G;
 
-  uint32_t primed = 0;
   if (tid == 0) {
     for (int s = 0; s < SW; ++s) { mbar_init(&w_full[s], 1); mbar_init(&w_empty[s], 4); }
     for (int s = 0; s < SC; ++s) { mbar_init(&c_full[s], 1); mbar_init(&c_empty[s], ISSUERS); }
@@ -229,18 +228,21 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     for (int b = 0; b < 2; ++b) { mbar_init(&d_full[b], ISSUERS); mbar_init(&d_empty[b], 4); }
     abort_flag_s = 0;
     mbar_fence_init();
-    // The packed weights depend on no earlier kernel: the first ring-full of copies leaves before
-    // the CTA has even allocated its tensor memory, and (programmatic dependent launch) while the
-    // kernel that quantizes the activations may still be running.
-    Range range(p, u0, u1);
-    Segment sg;
-    while (primed < (uint32_t)SW && range.next(sg)) {
-      const Job& job = p.jobs[sg.job];
-      for (int kb = sg.ka; kb < sg.ke && primed < (uint32_t)SW; ++kb, ++primed) {
-        mbar_expect_tx(&w_full[primed], W_BYTES);
-        bulk_load(w_ring + (size_t)primed * W_BYTES, job.Wp + ((size_t)sg.rb * job.n_kb + kb) * W_BYTES, W_BYTES,
-                  &w_full[primed]);
-      }
+  }
+  // The packed weights depend on no earlier kernel: the first ring-full of copies leaves before
+  // the CTA has even allocated its tensor memory, and (programmatic dependent launch) while the
+  // kernel that quantizes the activations may still be running.  Lane l of warp 0 issues stage l's.
+  const uint32_t primed = (u1 - u0) < (uint32_t)SW ? (u1 - u0) : (uint32_t)SW;
+  if (warp == 0) {
+    __syncwarp();
+    if ((uint32_t)lane < primed) {
+      const uint32_t u = u0 + (uint32_t)lane;
+      int j = 0;
+      while (j + 1 < p.n_jobs && u >= p.jobs[j + 1].u_begin) ++j;
+      const Job& job = p.jobs[j];
+      mbar_expect_tx(&w_full[lane], W_BYTES);
+      // units of a job lie in memory in the order they are numbered
+      bulk_load(w_ring + (size_t)lane * W_BYTES, job.Wp + (size_t)(u - job.u_begin) * W_BYTES, W_BYTES, &w_full[lane]);
     }
   }
   if (warp == 1) {
@@ -465,7 +467,7 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
         // Everything that needs neither the accumulators nor the other CTAs' parts happens before the
         // wait: this segment is the CTA's last, so what follows it is the tail of the whole kernel.
         own_o = o; own_tok0 = tok0;
-        while (c + 1 + n_follow < G && U * (c + 1 + n_follow) / G < sg.rb_end) ++n_follow;
+        while (c + 1 + n_follow < G && U * (uint32_t)(c + 1 + n_follow) / (uint32_t)G < sg.rb_end) ++n_follow;
       }
       ok = ok && warp_wait<true>(&d_full[b], (seg >> 1) & 1, abort_flag, p.status);
       ++seg;
@@ -681,11 +683,12 @@ static int launch_gemm_stream_pass(const StreamInput* inputs, int n_inputs, cons
     jb.scale = in.scale; jb.codesum = in.codesum; jb.alpha = jobs[j].alpha;
     jb.y = jobs[j].y; jb.acc_out = jobs[j].acc_out;
     jb.N = jobs[j].N; jb.n_kb = in.K / (128 * kbp); jb.map = jobs[j].input;
-    jb.u_begin = u;
+    jb.u_begin = (uint32_t)u;
     u += (long)((jobs[j].N + 127) / 128) * jb.n_kb;
   }
   for (int j = n_jobs; j < MAX_JOBS; ++j) p.jobs[j] = p.jobs[0];
-  p.U = u;
+  if (u > (long)(0xFFFFFFFFu / (MAX_GRID + 1))) return HBL_ERR_TOO_LARGE;   // the kernel indexes units in 32 bits
+  p.U = (uint32_t)u;
   p.part = part; p.flags = flags;
   p.status = device_status_word();
   if (p.status == nullptr) return HBL_ERR_CUDA;
