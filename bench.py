@@ -40,7 +40,7 @@ L2_BYTES = 126 * 1024 * 1024
 RING_BYTES = 4 * L2_BYTES            # ring of distinct input sets so that every call is L2-cold
 NOMINAL_INT8_TOPS = 4500.0
 ALU_PEAK_LANE_OPS = 148 * 128 * 1.965e9      # fp32 lanes x SMs x clocks.max.sm
-GEMM_TENSOR_TRAFFIC_BYTES = 194903552        # 151.11 MB read + 43.79 MB written per launch (headline workload)
+GEMM_TENSOR_TRAFFIC_BYTES = 205914112        # 156.23 MB read + 49.68 MB written per launch (headline workload)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
