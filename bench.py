@@ -223,6 +223,34 @@ def layer_point(name, kind, seed, K, N, bits, had, T, torch, hbl, peaks, iters=N
     return out
 
 
+def backward_transform_point(K, T, torch, hbl, peaks, iters=None):
+    """The transform's backward pass (the same orthonormal product on a bf16 gradient, bf16 out): bound by
+    HBM, 4 B per element.  L2-cold: a ring of distinct gradient buffers larger than L2."""
+    per_call = 4 * T * K
+    ring = max(2, min(16, -(-RING_BYTES // per_call)))
+    gen = torch.Generator(device="cuda").manual_seed(900 + K)
+    gs = [torch.randn((T, K), device="cuda", generator=gen).bfloat16() for _ in range(ring)]
+    outs = [torch.empty_like(g) for g in gs]
+    state = {"i": 0}
+
+    def call():
+        r = state["i"] % ring
+        state["i"] += 1
+        hbl.hbl_hadamard_bf16(gs[r], outs[r])
+
+    ms = time_loop(call, iters or 30, 3, torch)
+    st = hbl.hbl_check_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} in backward transform K={K}")
+    gbs = per_call / (ms * 1e-3) / 1e9
+    out = {"point": "transform_backward_bf16", "tokens": T, "in": K, "out": K, "bits": 16, "hadamard": True,
+           "ms": round(ms, 5), "tokens_per_s": round(T / (ms * 1e-3), 1), "tops": 0.0, "alg_gbs": round(gbs, 1),
+           "ring": ring, "graph": False, "bound": "hbm", "frac": round(gbs / peaks["hbm_gbs"], 4)}
+    del gs, outs
+    torch.cuda.empty_cache()
+    return out
+
+
 def block_point(T, torch, hbl, peaks, iters=None):
     """7B-shaped decoder-block projection sweep point (config 5)."""
     from paper_2504_18415_b200 import workloads as wl
@@ -498,6 +526,10 @@ def main():
         for N_ in (12288, 32768):
             for T_ in ((16, 4096, 32768) if full else (16, 4096)):
                 L(f"config4_a8_N{N_}", "gauss", 4, 4096, N_, 8, False, T_)
+        if full:
+            for K_ in (4096, 8192):
+                if want("transform_backward_bf16", 16384):
+                    points.append(backward_transform_point(K_, 16384, torch, hbl, peaks))
         for T_ in ((1, 4, 16, 64, 256, 1024, 4096, 16384, 65536) if full else (1, 16, 256, 4096)):
             if want("config5_block_7B", T_):
                 points.append(block_point(T_, torch, hbl, peaks))

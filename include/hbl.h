@@ -146,6 +146,15 @@ int hbl_check_status(void* stream);
 /* Eq. 3-4 alone: xr_out[T,K] fp32 = H_m x, orthonormal, natural order. */
 int hbl_hadamard_f32(const void* x, int x_dtype, int tokens, int in_dim, float* xr_out, void* stream);
 
+/* The transform alone with bf16 in and bf16 out, for the backward pass: the gradient with respect to
+ * the layer input is the same orthonormal transform applied to the gradient with respect to the
+ * transformed input (section 2.2 "Training", the equation after Eq. 7; H_m is symmetric and its own
+ * inverse).  out[T,K] = H_m g, natural order, fp32 arithmetic, one rounding to bf16 at the end.
+ *   g, out   device, bf16 [tokens, in_dim] row-major, 16-byte aligned, caller-owned; may not alias.
+ *   in_dim   2048, 4096, 8192 or 16384 (HBL_ERR_NOT_POW2 / HBL_ERR_SHAPE otherwise); tokens >= 0.
+ * Asynchronous on `stream`; returns a status code, allocates nothing. */
+int hbl_hadamard_bf16(const void* g, int tokens, int in_dim, void* out, void* stream);
+
 /* Eq. 3-6: transform (optional), per-token statistic, quantize.  codes_out: int8
  * [T,K], one code per byte; scale_out: fp32 [T] (s_t); codesum_out: int32 [T],
  * sum_k q[t,k] (may be NULL). */

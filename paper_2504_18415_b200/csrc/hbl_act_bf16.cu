@@ -285,6 +285,41 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   }
 
   constexpr float norm = G::NORM;
+  if constexpr (BITS == 0) {
+    // Transform only, bf16 out (the backward pass of the transform, Eq. 8, is this same product applied
+    // to the gradient): `codes` is the bf16 output [T, K].  One rounding, fp32 -> bf16, after the scale.
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(codes) + token * K;
+    if (live) {
+      if constexpr (C == 0) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          float lo, hi;
+          unpack2(v[e], lo, hi);
+          out[findex(2 * e)] = __float2bfloat16_rn(lo * norm);
+          out[findex(2 * e + 1)] = __float2bfloat16_rn(hi * norm);
+        }
+      } else {
+        constexpr int PAIRS = RUN / 2;                       // pairs per run of consecutive elements
+#pragma unroll
+        for (int r = 0; r < 32 / PAIRS; ++r) {
+          uint32_t w[PAIRS];
+#pragma unroll
+          for (int q = 0; q < PAIRS; ++q) {
+            float lo, hi;
+            unpack2(v[r * PAIRS + q], lo, hi);
+            const __nv_bfloat162 h = __floats2bfloat162_rn(lo * norm, hi * norm);
+            w[q] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+          __nv_bfloat16* dst = out + findex(r * RUN);
+          if constexpr (PAIRS == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+          else if constexpr (PAIRS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+          else *reinterpret_cast<uint32_t*>(dst) = w[0];
+        }
+      }
+    }
+    grid_dependency_wait();
+    return;
+  }
   if (xr_out != nullptr) {       // stage export (uniform over the grid): x_r in fp32, nothing else
     if (live) {
 #pragma unroll
@@ -428,6 +463,18 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
 }
 
 }  // namespace
+
+int launch_hadamard_bf16(const void* x, int T, int K, void* out, cudaStream_t s) {
+  if (T <= 0) return HBL_OK;
+  int8_t* o = static_cast<int8_t*>(out);
+  switch (K) {
+    case 2048: return launch_one<11, 0>(x, T, 1.0f, o, nullptr, nullptr, nullptr, nullptr, 0, s);
+    case 4096: return launch_one<12, 0>(x, T, 1.0f, o, nullptr, nullptr, nullptr, nullptr, 0, s);
+    case 8192: return launch_one<13, 0>(x, T, 1.0f, o, nullptr, nullptr, nullptr, nullptr, 0, s);
+    case 16384: return launch_one<14, 0>(x, T, 1.0f, o, nullptr, nullptr, nullptr, nullptr, 0, s);
+    default: return HBL_ERR_SHAPE;
+  }
+}
 
 bool act_quant_bf16_supported(int K) { return K == 2048 || K == 4096 || K == 8192 || K == 16384; }
 

@@ -343,6 +343,17 @@ int hbl_hadamard_f32(const void* x, int x_dtype, int tokens, int in_dim, float* 
                           static_cast<cudaStream_t>(stream));
 }
 
+int hbl_hadamard_bf16(const void* g, int tokens, int in_dim, void* out, void* stream) {
+  int rc = check_dims(tokens, in_dim, 16);
+  if (rc != HBL_OK) return rc;
+  if (!is_pow2(in_dim)) return HBL_ERR_NOT_POW2;
+  if (in_dim < 2048 || in_dim > 16384) return HBL_ERR_SHAPE;
+  if (tokens == 0) return HBL_OK;
+  if (!g || !out) return HBL_ERR_NULL;
+  if (!aligned(g, 16) || !aligned(out, 16)) return HBL_ERR_ALIGN;
+  return launch_hadamard_bf16(g, tokens, in_dim, out, static_cast<cudaStream_t>(stream));
+}
+
 int hbl_quantize_act(const void* x, int x_dtype, int tokens, int in_dim, int bits, int use_hadamard,
                      float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out, void* stream) {
   int rc = check_dims(tokens, in_dim, 16);

@@ -25,7 +25,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "hbl_status_string", "hbl_packed_weight_bytes", "hbl_workspace_bytes",
     "hbl_quantize_weights_workspace_bytes", "hbl_quantize_weights", "hbl_forward",
-    "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32",
+    "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16",
     "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
     "hbl_profile_events", "hbl_gemm_i32_static",
 ]
@@ -70,6 +70,7 @@ def lib() -> C.CDLL:
         L.hbl_block_forward.argtypes = [C.POINTER(hbl_block_t), vp, sz, i, vp]
         L.hbl_check_status.argtypes = [vp]
         L.hbl_hadamard_f32.argtypes = [vp, i, i, i, vp, vp]
+        L.hbl_hadamard_bf16.argtypes = [vp, i, i, vp, vp]
         L.hbl_quantize_act.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp]
         L.hbl_gemm_i32.argtypes = [vp, vp, i, i, vp, i, vp, vp, sz, i, vp]
         L.hbl_unpack_weights.argtypes = [vp, i, i, vp, vp]
@@ -82,7 +83,7 @@ def lib() -> C.CDLL:
         L.hbl_profile_events.argtypes = [C.POINTER(vp), C.POINTER(vp), i, i]
         L.hbl_profile_events.restype = C.c_int
         for n in ("hbl_quantize_weights", "hbl_forward", "hbl_block_forward", "hbl_check_status",
-                  "hbl_hadamard_f32", "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights"):
+                  "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -196,6 +197,15 @@ def hbl_hadamard_f32(x: torch.Tensor) -> torch.Tensor:
     T, K = x.shape
     out = torch.empty((T, K), dtype=torch.float32, device=x.device)
     _check(lib().hbl_hadamard_f32(_ptr(x), _dt(x), T, K, _ptr(out), _stream()), "hbl_hadamard_f32")
+    return out
+
+
+def hbl_hadamard_bf16(g: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """bf16 [T,K] -> bf16 [T,K]: the orthonormal transform alone (the backward pass applies it to the gradient)."""
+    T, K = g.shape
+    if out is None:
+        out = torch.empty((T, K), dtype=torch.bfloat16, device=g.device)
+    _check(lib().hbl_hadamard_bf16(_ptr(g), T, K, _ptr(out), _stream()), "hbl_hadamard_bf16")
     return out
 
 

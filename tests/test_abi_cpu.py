@@ -67,6 +67,10 @@ def test_argument_errors_come_before_any_launch(L):
     assert q(p, 0, 512, 512, -1.0, p, p, p, 1 << 20, n) == 7
     assert q(p, 0, 512, 512, 1e-5, p, p, p, 8, n) == 6
     assert L.hbl_hadamard_f32(p, 0, 4, 384, p, n) == 3
+    assert L.hbl_hadamard_bf16(p, 4, 384, p, n) == 3             # not a power of two
+    assert L.hbl_hadamard_bf16(p, 4, 1024, p, n) == 2            # outside 2048..16384
+    assert L.hbl_hadamard_bf16(n, 4, 4096, p, n) == 1
+    assert L.hbl_hadamard_bf16(p, 0, 4096, p, n) == 0            # no tokens: no-op
     assert L.hbl_quantize_act(p, 0, 4, 512, 3, 1, 1e-5, p, p, p, n) == 4
     assert L.hbl_gemm_i32(p, n, 4, 512, p, 512, p, p, 1 << 30, hbl.PATH_STREAM, n) == 1   # codesum required
     b = hbl.hbl_block_t()

@@ -44,6 +44,44 @@ def test_hadamard_unit_vectors_and_involution():
     assert np.allclose(back, y, atol=1e-5 * np.abs(y).max())
 
 
+@pytest.mark.parametrize("K", [2048, 4096, 8192, 16384])
+def test_hadamard_bf16_backward_matches_oracle(K):
+    """The backward pass of the transform (the equation after Eq. 7 in the training section): the same
+    orthonormal product applied to the gradient, bf16 in and out.  The oracle's transform in fp64 is the
+    reference; the kernel computes in fp32 and rounds once to bf16, so an output may differ from the exact
+    value by half a bf16 ulp (2^-9 relative) plus the fp32 error of log2 K butterfly stages, bounded here
+    by 2^-18 of the row's largest output."""
+    T = 37 if K <= 8192 else 9
+    g = wl.rows("gauss", 300 + K, 1, K, 0, T, "bf16")
+    got = hbl.hbl_hadamard_bf16(to_dev(g, "bf16")).float().cpu().numpy().astype(np.float64)
+    want = orc.hadamard(g)
+    tol = 2.0 ** -8 * np.abs(want) + 2.0 ** -18 * np.abs(want).max(axis=1, keepdims=True)
+    assert np.all(np.abs(got - want) <= tol), float((np.abs(got - want) / tol).max())
+
+
+def test_hadamard_bf16_exact_cases_and_involution():
+    K = 8192                                   # 1/sqrt(K) is not a power of two here: one rounding in the scale
+    x = np.zeros((3, K), np.float32)
+    x[0, 5] = 1; x[1, :] = 1; x[2, 0] = 3; x[2, 1] = -3
+    got = hbl.hbl_hadamard_bf16(to_dev(x, "bf16")).float().cpu().numpy()
+    s = np.float32(1.0 / np.sqrt(np.float64(K)))
+    sb = torch.tensor([s]).bfloat16().float().item()
+    idx = np.arange(K)
+    par5 = np.array([bin(i & 5).count("1") & 1 for i in idx])
+    assert np.array_equal(got[0], np.where(par5, -sb, sb).astype(np.float32))          # column 5 of H, up to sign
+    assert got[1, 0] == torch.tensor([K * s]).bfloat16().float().item() and np.all(got[1, 1:] == 0)
+    want2 = np.where(idx & 1, 6 * s, 0).astype(np.float32)                              # 3 e0 - 3 e1
+    assert np.array_equal(got[2], torch.from_numpy(want2).bfloat16().float().numpy())
+    # applied twice it is the identity, up to the two bf16 roundings
+    y = wl.rows("gauss", 2, 1, K, 0, 8, "bf16")
+    yd = to_dev(y, "bf16")
+    back = hbl.hbl_hadamard_bf16(hbl.hbl_hadamard_bf16(yd)).float().cpu().numpy()
+    assert np.all(np.abs(back - y) <= 2.0 ** -7 * np.abs(y).max())
+    # and it agrees with the fp32 export of the forward kernel, rounded
+    f32 = hbl.hbl_hadamard_f32(yd)
+    assert torch.equal(hbl.hbl_hadamard_bf16(yd), f32.bfloat16())
+
+
 @pytest.mark.parametrize("K", ALL_K)
 @pytest.mark.parametrize("bits", [4, 8])
 @pytest.mark.parametrize("had", [True, False])
