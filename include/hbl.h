@@ -119,6 +119,12 @@ int hbl_block_forward(const hbl_block_t* block /* host pointer */, void* workspa
  * to be asynchronous): copies x_host -> x_stage, runs the layer, copies y_stage ->
  * y_host, all enqueued on `stream`.  x_stage / y_stage are DEVICE staging buffers
  * of tokens*in_dim*sizeof(x) and tokens*out_dim*2 bytes owned by the caller.
+ * Calls of more than 2048 tokens run as a pipeline over chunks of tokens (rows are
+ * independent): one chunk is copied in, one computed, one copied out at a time, on
+ * the caller's stream and two side streams that the library creates on its first
+ * such call on a device (so that first call should come before any stream capture).
+ * In the caller's stream order the call is complete when y_host is; workspace as
+ * for hbl_forward with max_tokens = tokens.  Results are those of hbl_forward.
  * No counterpart in the paper beyond Eq. 3-7 themselves. */
 int hbl_forward_host(const void* x_host /* host */, int x_dtype, int tokens, int in_dim,
                      const void* W_packed, const float* alpha, int out_dim, int bits, int use_hadamard,

@@ -302,6 +302,37 @@ int hbl_profile_events(void** start_events, void** stop_events, int n, int kerne
   return used;
 }
 
+namespace {
+
+// Side streams and events of hbl_forward_host, created on first use, one set per device.
+constexpr int kHostMaxChunks = 16;
+constexpr int kHostChunkTokens = 2048;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t start = nullptr, out_done = nullptr, in_done[kHostMaxChunks] = {}, comp_done[kHostMaxChunks] = {};
+};
+HostPipe* host_pipe() {
+  static HostPipe pipes[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostPipe& hp = pipes[dev];
+  if (!hp.ready) {
+    if (cudaStreamCreateWithFlags(&hp.copy_in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&hp.copy_out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    for (int c = 0; c < kHostMaxChunks; ++c) {
+      if (cudaEventCreateWithFlags(&hp.in_done[c], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&hp.comp_done[c], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    hp.ready = true;
+  }
+  return &hp;
+}
+
+}  // namespace
+
 int hbl_forward_host(const void* x_host, int x_dtype, int tokens, int in_dim, const void* W_packed,
                      const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y_host,
                      void* x_stage, void* y_stage, void* workspace, size_t workspace_bytes, int path,
@@ -309,14 +340,48 @@ int hbl_forward_host(const void* x_host, int x_dtype, int tokens, int in_dim, co
   if (tokens < 0) return HBL_ERR_SHAPE;
   if (tokens > 0 && (!x_host || !y_host || !x_stage || !y_stage)) return HBL_ERR_NULL;
   if (x_dtype != HBL_F32 && x_dtype != HBL_BF16) return HBL_ERR_FORMAT;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const size_t xb = (size_t)tokens * in_dim * (x_dtype == HBL_F32 ? 4 : 2);
-  const size_t yb = (size_t)tokens * out_dim * 2;
-  if (tokens > 0) HBL_CUDA_OK(cudaMemcpyAsync(x_stage, x_host, xb, cudaMemcpyHostToDevice, s));
-  int rc = hbl_forward(x_stage, x_dtype, tokens, in_dim, W_packed, alpha, out_dim, bits, use_hadamard, eps,
-                       y_stage, workspace, workspace_bytes, path, stream);
+  int rc = check_dims(tokens, in_dim, out_dim);
   if (rc != HBL_OK) return rc;
-  if (tokens > 0) HBL_CUDA_OK(cudaMemcpyAsync(y_host, y_stage, yb, cudaMemcpyDeviceToHost, s));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t x_row = (size_t)in_dim * (x_dtype == HBL_F32 ? 4 : 2), y_row = (size_t)out_dim * 2;
+  if (tokens <= kHostChunkTokens) {
+    // small calls: copy in, run, copy out, all in order on the caller's stream
+    if (tokens > 0) HBL_CUDA_OK(cudaMemcpyAsync(x_stage, x_host, x_row * tokens, cudaMemcpyHostToDevice, s));
+    rc = hbl_forward(x_stage, x_dtype, tokens, in_dim, W_packed, alpha, out_dim, bits, use_hadamard, eps,
+                     y_stage, workspace, workspace_bytes, path, stream);
+    if (rc != HBL_OK) return rc;
+    if (tokens > 0) HBL_CUDA_OK(cudaMemcpyAsync(y_host, y_stage, y_row * tokens, cudaMemcpyDeviceToHost, s));
+    return HBL_OK;
+  }
+  // Large calls run as a pipeline over chunks of tokens (rows are independent, Eq. 3-7 are per token):
+  // chunk c+1 crosses the bus on one side stream while chunk c is computed on the caller's stream and
+  // chunk c-1 returns on the other side stream, so the call costs about what its larger copy costs.
+  HostPipe* hp = host_pipe();
+  if (hp == nullptr) return HBL_ERR_CUDA;
+  int chunk = kHostChunkTokens;
+  if ((tokens + chunk - 1) / chunk > kHostMaxChunks) chunk = ((tokens + kHostMaxChunks - 1) / kHostMaxChunks + 127) / 128 * 128;
+  const int n_chunks = (tokens + chunk - 1) / chunk;
+  HBL_CUDA_OK(cudaEventRecord(hp->start, s));                 // what the caller queued before (it may still use the stages)
+  HBL_CUDA_OK(cudaStreamWaitEvent(hp->copy_in, hp->start, 0));
+  HBL_CUDA_OK(cudaStreamWaitEvent(hp->copy_out, hp->start, 0));
+  for (int c = 0; c < n_chunks; ++c) {
+    const int t0 = c * chunk, tn = tokens - t0 < chunk ? tokens - t0 : chunk;
+    const char* xh = static_cast<const char*>(x_host) + x_row * t0;
+    char* xd = static_cast<char*>(x_stage) + x_row * t0;
+    char* yd = static_cast<char*>(y_stage) + y_row * t0;
+    char* yh = static_cast<char*>(y_host) + y_row * t0;
+    HBL_CUDA_OK(cudaMemcpyAsync(xd, xh, x_row * tn, cudaMemcpyHostToDevice, hp->copy_in));
+    HBL_CUDA_OK(cudaEventRecord(hp->in_done[c], hp->copy_in));
+    HBL_CUDA_OK(cudaStreamWaitEvent(s, hp->in_done[c], 0));
+    rc = hbl_forward(xd, x_dtype, tn, in_dim, W_packed, alpha, out_dim, bits, use_hadamard, eps, yd, workspace,
+                     workspace_bytes, path, stream);
+    if (rc != HBL_OK) return rc;
+    HBL_CUDA_OK(cudaEventRecord(hp->comp_done[c], s));
+    HBL_CUDA_OK(cudaStreamWaitEvent(hp->copy_out, hp->comp_done[c], 0));
+    HBL_CUDA_OK(cudaMemcpyAsync(yh, yd, y_row * tn, cudaMemcpyDeviceToHost, hp->copy_out));
+  }
+  HBL_CUDA_OK(cudaEventRecord(hp->out_done, hp->copy_out));
+  HBL_CUDA_OK(cudaStreamWaitEvent(s, hp->out_done, 0));       // the call is complete, in the caller's stream order, when y_host is
   return HBL_OK;
 }
 

@@ -143,3 +143,25 @@ def test_block_full_size_repeated_calls_agree(T):
             assert hbl.hbl_check_status() == 0, f"bounded wait ran out in call {it}"
             for n in ref:
                 assert torch.equal(outs[n], ref[n]), f"output {n} of call {it} differs"
+
+
+@pytest.mark.parametrize("T", [100, 5000])
+def test_forward_host_equals_forward(T):
+    """hbl_forward_host (pinned host x and y; above 2048 tokens a pipeline of token chunks over the caller's
+    stream and two side streams) returns exactly what hbl_forward returns on the same rows, call after call."""
+    K, N = 2048, 1040
+    x = wl.rows("attn_out", 77, 1, K, 0, T, "bf16")
+    W = wl.rows("latent", 77, 2, K, 0, N, "f32")
+    packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), EPS)
+    xd = to_dev(x, "bf16")
+    want = hbl.hbl_forward(xd, packed, alpha, N, 4, True, EPS).cpu()
+    xh = xd.cpu().pin_memory()
+    yh = torch.zeros((T, N), dtype=torch.bfloat16).pin_memory()
+    xs, ys = torch.empty_like(xd), torch.empty((T, N), dtype=torch.bfloat16, device="cuda")
+    work = hbl.new_workspace(hbl.hbl_workspace_bytes(T, K, N))
+    for _ in range(3):
+        yh.zero_()
+        hbl.hbl_forward_host(xh, packed, alpha, N, 4, True, yh, xs, ys, work)
+        torch.cuda.current_stream().synchronize()      # the caller's stream alone: it waits for the side streams
+        assert hbl.hbl_check_status() == 0
+        assert torch.equal(yh, want)
