@@ -54,6 +54,23 @@ def test_extreme_codes_do_not_overflow():
     assert np.all(got == 128 * K)
 
 
+@pytest.mark.parametrize("T", [16, 100])
+def test_stream_kernel_largest_accumulators(T):
+    """The small-batch kernel feeds the tensor core 64 (w + 1), so its accumulators are 64 times the sums of
+    Eq. 7 plus 64 times the code sums: the largest they can get is at the longest row the library accepts,
+    all weights +1 and all codes -128 (or 127)."""
+    K, N = 32768, 144
+    W = np.full((N, K), 1.0, np.float32)
+    packed, _ = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), EPS)
+    q = np.full((T, K), -128, np.int8)
+    q[1::2] = 127
+    qd = torch.from_numpy(q).cuda()
+    got = hbl.hbl_gemm_i32(qd, qd.to(torch.int32).sum(1, dtype=torch.int32), packed, N, hbl.PATH_STREAM).cpu().numpy()
+    assert hbl.hbl_check_status() == 0
+    want = q.astype(np.int64).sum(1, keepdims=True).repeat(N, 1)
+    assert np.array_equal(got, want)
+
+
 def test_both_kernels_agree_and_runs_are_deterministic():
     T, K, N = 48, 4096, 4096
     q, packed, wt = setup(T, K, N, 4, 99)
