@@ -90,7 +90,12 @@ int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_
  *   bits      4 (Eq. 6) or 8 (Eq. 5);  use_hadamard: 1 applies Eq. 3-4 first
  *   y         [tokens, out_dim] bf16 (written)
  *   path      an hbl_path_t
- * The intermediate codes never leave the workspace. */
+ * The intermediate codes never leave the workspace.  On the large-batch path the
+ * packed weights are expanded to int8 (into the workspace) on a side stream of the
+ * library's, which forks from `stream` at the start of the call and joins it again
+ * before the contraction: in `stream`'s order the call is complete when y is.  The
+ * side stream is created by the first such call on a device (hbl_block_forward
+ * shares it), so that call should come before any stream capture. */
 int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim,
                 const void* W_packed, const float* alpha, int out_dim,
                 int bits, int use_hadamard, float eps, void* y,

@@ -97,6 +97,34 @@ int resolve_path(int path, int tokens, size_t packed_bytes) {
   return -2;
 }
 
+// A side stream per device on which the large-batch path expands packed weights to int8 while the
+// caller's stream quantizes activations or runs the previous contraction (the expansion is bound by
+// HBM, the contraction by the tensor cores, the quantizer by instruction issue: they overlap well).
+// Created on first use; every use forks from the caller's stream and joins it again before returning,
+// so in the caller's stream order a call is complete when its last kernel is.
+constexpr int kSideEvents = 16;
+struct SidePipe {
+  bool ready = false;
+  cudaStream_t side = nullptr;
+  cudaEvent_t fork = nullptr, unpacked[kSideEvents] = {}, consumed[kSideEvents] = {};
+};
+SidePipe* side_pipe() {
+  static SidePipe pipes[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  SidePipe& sp = pipes[dev];
+  if (!sp.ready) {
+    if (cudaStreamCreateWithFlags(&sp.side, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&sp.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    for (int i = 0; i < kSideEvents; ++i) {
+      if (cudaEventCreateWithFlags(&sp.unpacked[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&sp.consumed[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    sp.ready = true;
+  }
+  return &sp;
+}
+
 // quantized activations -> one projection.  Exactly one of y / acc_out set.
 int run_gemm(int path, const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
              const void* W_packed, int N, const float* alpha, void* y, int32_t* acc_out, int32_t* acc_ws,
@@ -184,14 +212,32 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
   int32_t* codesum = reinterpret_cast<int32_t*>(ws + w.codesum);
   int8_t* codes = reinterpret_cast<int8_t*>(ws + w.codes);
   const bool stream_path = (p == HBL_PATH_STREAM);
+  SidePipe* sp = nullptr;
+  int8_t* w_i8 = reinterpret_cast<int8_t*>(ws + w.w_i8);
+  if (!stream_path) {
+    // the weights are expanded on the side stream while the activations are quantized on the caller's
+    sp = side_pipe();
+    if (sp == nullptr) return HBL_ERR_CUDA;
+    HBL_CUDA_OK(cudaEventRecord(sp->fork, s));
+    HBL_CUDA_OK(cudaStreamWaitEvent(sp->side, sp->fork, 0));
+    rc = launch_unpack_weights(W_packed, out_dim, in_dim, w_i8, sp->side);
+    if (rc != HBL_OK) return rc;
+    HBL_CUDA_OK(cudaEventRecord(sp->unpacked[0], sp->side));
+  }
   rc = launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale,
                         stream_path ? codesum : nullptr /* only the streaming kernel needs the code sums */, nullptr,
                         stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
                         stream_path ? w.zero_words : 0, s);
-  if (rc != HBL_OK) return rc;
-  return run_gemm(p, codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha, y, nullptr,
-                  reinterpret_cast<int32_t*>(ws + w.acc), reinterpret_cast<int*>(ws + w.counters),
-                  reinterpret_cast<int8_t*>(ws + w.w_i8), s);
+  if (rc != HBL_OK) {
+    if (sp != nullptr) cudaStreamWaitEvent(s, sp->unpacked[0], 0);   // join before reporting the error
+    return rc;
+  }
+  if (stream_path)
+    return launch_gemm_stream(codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha,
+                              static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
+                              reinterpret_cast<int*>(ws + w.counters), s);
+  HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[0], 0));
+  return launch_gemm_tensor(codes, scale, tokens, in_dim, w_i8, out_dim, alpha, static_cast<__nv_bfloat16*>(y), nullptr, s);
 }
 
 // ---- decoder block: four quantizations, seven projections -------------------------------
@@ -213,7 +259,7 @@ BlockWs carve_block(int T, int H, int F) {
   for (int i = 0; i < 7; ++i) { w.acc[i] = off; off += sizeof(int32_t) * gemm_stream_acc_words(ts, out_dims[i]); }
   off = align_up(off, 1024);
   for (int i = 0; i < 4; ++i) { w.codes[i] = off; off = align_up(off + (size_t)T * in_dims[i], 1024); }
-  w.w_i8 = off; off = align_up(off + (size_t)F * H, 1024);   // largest weight: F x H
+  w.w_i8 = off; off = align_up(off + 2 * align_up((size_t)F * H, 1024), 1024);   // two buffers of the largest weight (F x H)
   w.total = off;
   return w;
 }
@@ -258,6 +304,15 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   const int in_dims[4] = {H, H, H, F};
   const int had[4] = {0, 1, 0, 1};
   const bool stream_path = (p == HBL_PATH_STREAM);
+  SidePipe* sp = nullptr;
+  if (!stream_path) {
+    // fork the side stream now: its first expansions overlap the quantizations below, and it starts
+    // after whatever the caller queued before (an earlier call may still be reading the int8 buffers)
+    sp = side_pipe();
+    if (sp == nullptr) return HBL_ERR_CUDA;
+    HBL_CUDA_OK(cudaEventRecord(sp->fork, s));
+    HBL_CUDA_OK(cudaStreamWaitEvent(sp->side, sp->fork, 0));
+  }
   for (int i = 0; i < 4; ++i) {
     rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
                           reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
@@ -280,15 +335,23 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, reinterpret_cast<int32_t*>(ws + w.acc[0]),
                                     reinterpret_cast<int*>(ws + w.counters[0]), s);
   }
-  for (int i = 0; i < 7; ++i) {
+  // Large batch: tensor i+1 is expanded to int8 on the side stream (two buffers alternate) while tensor i
+  // is contracted on the caller's stream.
+  const size_t buf_bytes = align_up((size_t)F * H, 1024);
+  for (int i = 0; i < 7 && rc == HBL_OK; ++i) {
     const int xi = src[i];
-    rc = run_gemm(p, reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]),
-                  reinterpret_cast<int32_t*>(ws + w.codesum[xi]), T, in_dims[xi], Ws[i], out_dims[i],
-                  b->alpha7 + i, ys[i], nullptr, reinterpret_cast<int32_t*>(ws + w.acc[i]),
-                  reinterpret_cast<int*>(ws + w.counters[i]), reinterpret_cast<int8_t*>(ws + w.w_i8), s);
-    if (rc != HBL_OK) return rc;
+    int8_t* w_i8 = reinterpret_cast<int8_t*>(ws + w.w_i8 + (size_t)(i & 1) * buf_bytes);
+    if (i >= 2) HBL_CUDA_OK(cudaStreamWaitEvent(sp->side, sp->consumed[i - 2], 0));   // the buffer's previous reader
+    rc = launch_unpack_weights(Ws[i], out_dims[i], in_dims[xi], w_i8, sp->side);
+    if (rc != HBL_OK) break;
+    HBL_CUDA_OK(cudaEventRecord(sp->unpacked[i], sp->side));
+    HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[i], 0));
+    rc = launch_gemm_tensor(reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]), T,
+                            in_dims[xi], w_i8, out_dims[i], b->alpha7 + i, static_cast<__nv_bfloat16*>(ys[i]), nullptr, s);
+    if (rc != HBL_OK) break;
+    HBL_CUDA_OK(cudaEventRecord(sp->consumed[i], s));
   }
-  return HBL_OK;
+  return rc;
 }
 
 unsigned long long hbl_launch_count(void) { return g_launches; }
