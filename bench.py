@@ -456,11 +456,17 @@ def main():
 
     # per-kernel breakdown (outside the timed region)
     breakdown = {}
-    for kid, name in ((1, "act_quant_kernel"), (3, "unpack_kernel"), (2, "gemm_tensor_kernel")):
+    for kid, name in ((1, "act_quant_kernel"), (2, "gemm_tensor_kernel")):
         with hbl.KernelTimer(5, kid) as k2:
             for i in range(5):
                 step(i)
         breakdown[name] = round(statistics.mean(k2.times_ms()), 5)
+    # Inside a step the weight expansion runs on the library's side stream underneath the quantizer, so its
+    # own duration is taken from stand-alone launches of the same kernel.
+    with hbl.KernelTimer(5, 3) as k2:
+        for i in range(5):
+            hbl.hbl_unpack_weights(packed, N, K)
+    breakdown["unpack_kernel"] = round(statistics.mean(k2.times_ms()), 5)
 
     if rank != 0:
         if dist is not None:
@@ -503,7 +509,8 @@ def main():
             "alu_frac": round(12.5 * T * K / (act_ms * 1e-3) / ALU_PEAK_LANE_OPS, 4),
             "note": "3 B of kernel traffic and 12.5 fp32 lane-ops per element; ALU peak 148 SMs x 128 lanes x 1.965 GHz"},
         "unpack_kernel": {"ms": breakdown["unpack_kernel"],
-                          "hbm_frac": round(1.25 * N * K / (breakdown["unpack_kernel"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)},
+                          "hbm_frac": round(1.25 * N * K / (breakdown["unpack_kernel"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                          "note": "timed alone; inside the step it overlaps the quantizer on a side stream"},
         "gemm_tensor_kernel": {"ms": breakdown["gemm_tensor_kernel"]},
     }
 
