@@ -83,13 +83,16 @@ int check_quant_args(int x_dtype, int in_dim, int bits, int use_hadamard, float 
   return HBL_OK;
 }
 
-// Which contraction kernel.  The streaming kernel reads the packed weights once per 128 tokens: up to
-// 128 tokens it always wins; up to 512 it wins when there are enough weight bytes for its fixed costs
-// to disappear (measured: a 7B block yes, a single 2048 x 2048 layer no).
-int resolve_path(int path, int tokens, size_t packed_bytes) {
+// Which contraction kernel.  The streaming kernel reads the packed weights once per 128 tokens; the
+// large-batch path pays an expansion and a launch per weight tensor.  Measured cross-overs: one pass
+// (<= 128 tokens) always goes to the streaming kernel; a single layer of 16 MiB or more of packed weights
+// up to 192 tokens (at 256 the two are level, beyond it the large-batch path wins: 32 MiB at 512 tokens
+// 161 vs 104 us); the seven tensors of a decoder block up to 512 tokens (64 MiB: 271 vs 268 us there).
+int resolve_path(int path, int tokens, size_t packed_bytes, int n_tensors) {
   if (path == HBL_PATH_AUTO) {
     if (tokens <= 128) return HBL_PATH_STREAM;
-    if (tokens <= kStreamMaxTokens && packed_bytes >= (size_t)16 << 20) return HBL_PATH_STREAM;
+    const int limit = n_tensors > 1 ? kStreamMaxTokens : 192;
+    if (tokens <= limit && packed_bytes >= (size_t)16 << 20) return HBL_PATH_STREAM;
     return HBL_PATH_TENSOR;
   }
   if (path == HBL_PATH_STREAM) return tokens <= kStreamMaxTokens ? HBL_PATH_STREAM : -1;
@@ -196,7 +199,7 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
   if (rc != HBL_OK) return rc;
   rc = check_quant_args(x_dtype, in_dim, bits, use_hadamard, eps);
   if (rc != HBL_OK) return rc;
-  const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4);
+  const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4, 1);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
   if (tokens == 0) return HBL_OK;
@@ -280,7 +283,7 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   rc = check_quant_args(b->x_dtype, H, b->bits, 1, b->eps);
   if (rc != HBL_OK) return rc;
   if (!is_pow2(F)) return HBL_ERR_NOT_POW2;
-  const int p = resolve_path(path, T, ((size_t)4 * H * H + (size_t)3 * H * F) / 4);
+  const int p = resolve_path(path, T, ((size_t)4 * H * H + (size_t)3 * H * F) / 4, 7);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
   if (T == 0) return HBL_OK;
@@ -499,7 +502,7 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
                  int out_dim, int32_t* acc_out, void* workspace, size_t workspace_bytes, int path, void* stream) {
   int rc = check_dims(tokens, in_dim, out_dim);
   if (rc != HBL_OK) return rc;
-  const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4);
+  const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4, 1);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
   if (tokens == 0) return HBL_OK;
