@@ -5,6 +5,7 @@
 // tcgen05.ld.
 //
 //   D[128 tokens, 256 weight rows] += A[128, 32] * B[256, 32]^T   per instruction
+//   (128 weight rows per tile on very small grids, see launch_gemm_tensor)
 //
 // Persistent, warp-specialised, one CTA per SM:
 //   warp 0      TMA producer: 4-stage ring of (A 128x128 B, B 256x128 B) tiles, 128-byte swizzle
@@ -25,22 +26,27 @@ namespace hbl {
 namespace {
 
 constexpr int BM = 128;              // tokens per tile (MMA M, TMEM lanes)
-constexpr int BN = 256;              // weight rows per tile (MMA N, TMEM columns)
 constexpr int BK = 128;              // bytes (= int8 elements) of K per stage: one swizzle atom
 constexpr int UMMA_K = 32;           // K of one kind::i8 instruction
-constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK;     // 16 KiB
-constexpr int B_BYTES = BN * BK;     // 32 KiB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024;   // + alignment slack
+// Weight rows per tile (MMA N, TMEM columns): 256 is the efficient shape; 128 is used when 256-row tiles
+// would leave half of the SMs without a tile (it doubles the number of tiles).
+template <int BN>
+struct Shape {
+  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int B_BYTES = BN * BK;                // 32 or 16 KiB
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024;   // + alignment slack
+  // Instruction descriptor (32 bit): D format s32 (2) at bits [4,6); A and B format
+  // signed 8-bit (1) at [7,10) and [10,13); both K-major (bits 15, 16 = 0);
+  // N >> 3 at [17,23); M >> 4 at [24,29).
+  static constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                                    ((uint32_t)(BM >> 4) << 24);
+};
+constexpr int MAX_STAGES = 6;
 
-// Instruction descriptor (32 bit): D format s32 (2) at bits [4,6); A and B format
-// signed 8-bit (1) at [7,10) and [10,13); both K-major (bits 15, 16 = 0);
-// N >> 3 at [17,23); M >> 4 at [24,29).
-constexpr uint32_t IDESC = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
-                           ((uint32_t)(BM >> 4) << 24);
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -104,11 +110,12 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, u
       : "memory");
 }
 
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
   asm volatile(
       "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
       " tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(IDESC), "r"(accumulate)
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -141,6 +148,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 // of the group at a time.  The CTAs that run at the same time then share a few weight tiles and a
 // few token blocks (both stay in L2) instead of sweeping the whole weight matrix per token block.
 constexpr int GROUP_M = 8;
+template <int BN>
 __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& m0, int& n0) {
   const int per_group = GROUP_M * tiles_n;
   const int first_m = (tile / per_group) * GROUP_M;
@@ -150,14 +158,16 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
   n0 = (local / gm) * BN;
 }
 
+template <int BN>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const float* __restrict__ scale, const float* __restrict__ alpha,
                    __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out, int T, int N, int K,
                    int* __restrict__ status) {
+  constexpr int STAGES = Shape<BN>::STAGES, STAGE_BYTES = Shape<BN>::STAGE_BYTES;
   extern __shared__ unsigned char smem_dyn[];
-  __shared__ __align__(8) uint64_t full_bar[STAGES];
-  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t tfull_bar[2];
   __shared__ __align__(8) uint64_t tempty_bar[2];
   __shared__ uint32_t tmem_slot;
@@ -193,7 +203,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         int m0, n0;
-        tile_coords(tile, tiles_m, tiles_n, m0, n0);
+        tile_coords<BN>(tile, tiles_m, tiles_n, m0, n0);
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abort_flag, status)) { ok = false; break; }
@@ -223,7 +233,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 #pragma unroll
           for (int ks = 0; ks < BK / UMMA_K; ++ks)
             umma_i8(d_tmem, adesc + (uint64_t)(ks * UMMA_K / 16), bdesc + (uint64_t)(ks * UMMA_K / 16),
-                    (kb | ks) != 0);
+                    Shape<BN>::IDESC, (kb | ks) != 0);
           umma_commit(&empty_bar[s]);          // stage reusable once these MMAs have read it
         }
         if (ok) umma_commit(&tfull_bar[b]);    // accumulator complete
@@ -237,7 +247,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tl) {
       const int b = tl & 1;
       int m0, n0;
-      tile_coords(tile, tiles_m, tiles_n, m0, n0);
+      tile_coords<BN>(tile, tiles_m, tiles_n, m0, n0);
       const bool got = mbar_wait(&tfull_bar[b], (tl >> 1) & 1, abort_flag, status);
       if (!__all_sync(0xffffffffu, got)) break;      // warp-uniform: tcgen05.ld needs the whole warp
       tc_fence_after();
@@ -324,33 +334,51 @@ int make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) 
   return r == CUDA_SUCCESS ? HBL_OK : HBL_ERR_CUDA;
 }
 
-}  // namespace
-
-int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
-                       const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s) {
-  if (T <= 0) return HBL_OK;
+template <int BN>
+int launch_shape(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N, const float* alpha,
+                 __nv_bfloat16* y, int32_t* acc_out, int n_sm, cudaStream_t s) {
   CUtensorMap tmA, tmB;
   int rc = make_map(&tmA, codes, T, K, BM);
   if (rc != HBL_OK) return rc;
   rc = make_map(&tmB, W_i8, N, K, BN);
   if (rc != HBL_OK) return rc;
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    HBL_CUDA_OK(cudaGetDevice(&dev));
-    HBL_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-    HBL_CUDA_OK(cudaFuncSetAttribute(gemm_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  static bool done = false;   // idempotent attribute; a race only repeats the call
+  if (!done) {
+    HBL_CUDA_OK(cudaFuncSetAttribute(gemm_tensor_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)Shape<BN>::SMEM_BYTES));
+    done = true;
   }
   int* status = device_status_word();
   if (status == nullptr) return HBL_ERR_CUDA;
   const int n_tiles = ((T + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
   profile_before(KERNEL_CONTRACT, s);
-  gemm_tensor_kernel<<<grid, THREADS, SMEM_BYTES, s>>>(tmA, tmB, scale, alpha, y, acc_out, T, N, K, status);
+  gemm_tensor_kernel<BN><<<grid, THREADS, Shape<BN>::SMEM_BYTES, s>>>(tmA, tmB, scale, alpha, y, acc_out, T, N, K, status);
   profile_after(KERNEL_CONTRACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
   return HBL_OK;
+}
+
+}  // namespace
+
+int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
+                       const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s) {
+  if (T <= 0) return HBL_OK;
+  static int n_sm = 0;
+  if (n_sm == 0) {
+    int dev = 0;
+    HBL_CUDA_OK(cudaGetDevice(&dev));
+    HBL_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  }
+  // The narrow tile only pays on very small grids, where even twice as many tiles leave half of the SMs
+  // idle (measured: 2048 x 2048 at 256 tokens 14.3 -> 12.8 us).  It costs about 1.5x per weight row (a
+  // 128 x 128 x 32 MMA reads as much of the token block from shared memory as a 128 x 256 x 32 one), and at
+  // larger sizes small-batch contractions are bound by L2 traffic, which narrower tiles increase
+  // (8192 -> 2048 at 1024 tokens: 37.6 -> 39.2 us; a 7B block at 4096 tokens: 0.96 -> 1.13 ms).
+  const long t128 = (long)((T + BM - 1) / BM) * ((N + 127) / 128);
+  if (N > 128 && 2 * t128 <= n_sm) return launch_shape<128>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
+  return launch_shape<256>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
 }
 
 }  // namespace hbl

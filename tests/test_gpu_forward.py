@@ -115,7 +115,7 @@ def test_block_full_size_repeated_calls_agree(T):
     shows only under some timings, so the same call is repeated and must give, every time, exactly the
     outputs of the first call and exactly those of the large-batch kernel (both contract exact integers and
     round once), with no bounded wait running out.  Weights are random ternary draws made on the device
-    (parity with the oracle at this size is covered by sampled outputs elsewhere)."""
+    (parity with the oracle at this size: sampled tokens in test_gpu_fullsize.py)."""
     cfg = wl.CONFIG5
     H, F = cfg.hidden, cfg.ffn
     g = torch.Generator(device="cuda").manual_seed(50 + T)
