@@ -217,6 +217,8 @@ def layer_point(name, kind, seed, K, N, bits, had, T, torch, hbl, peaks, iters=N
     else:
         out["bound"] = "tensor"
         out["frac"] = round(tops / (2 * peaks["bf16_tflops"]), 4)
+        # calls of a millisecond and more run under the power cap: the sustained figure is their ceiling
+        out["frac_of_sustained"] = round(tops / (2 * peaks["bf16_tflops_sustained"]), 4)
         out["frac_of_nominal_int8"] = round(tops / NOMINAL_INT8_TOPS, 4)
     del xs, ws, ys, work
     torch.cuda.empty_cache()
@@ -309,6 +311,7 @@ def block_point(T, torch, hbl, peaks, iters=None):
         out["bound"] = "hbm"; out["frac"] = round(gbs / peaks["hbm_gbs"], 4)
     else:
         out["bound"] = "tensor"; out["frac"] = round(tops / (2 * peaks["bf16_tflops"]), 4)
+        out["frac_of_sustained"] = round(tops / (2 * peaks["bf16_tflops_sustained"]), 4)
         out["frac_of_nominal_int8"] = round(tops / NOMINAL_INT8_TOPS, 4)
     del ins, sets, outs, work
     torch.cuda.empty_cache()
