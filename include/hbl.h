@@ -95,7 +95,9 @@ int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_
  * library's, which forks from `stream` at the start of the call and joins it again
  * before the contraction: in `stream`'s order the call is complete when y is.  The
  * side stream is created by the first such call on a device (hbl_block_forward
- * shares it), so that call should come before any stream capture. */
+ * shares it), so that call should come before any stream capture.  The side stream
+ * and its events are one set per device: issue large-batch calls for one device from
+ * one host thread at a time. */
 int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim,
                 const void* W_packed, const float* alpha, int out_dim,
                 int bits, int use_hadamard, float eps, void* y,
