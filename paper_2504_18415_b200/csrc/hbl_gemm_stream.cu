@@ -19,8 +19,8 @@
 //                 lane issues the MMAs; up to 32 token columns warps 1 and 3 issue half a unit each
 //   warps 4..11   unpack: two groups of four warps (one per TMEM lane quadrant) take alternate
 //                 units and hand the weight stage back as soon as its words are in registers
-//   warps 12..15  epilogue: read the accumulators (two D buffers alternate), subtract
-//                 the code sum (weights are fed as u = w + 1), rescale, store bf16
+//   warps 12..15  epilogue: read the accumulators (two D buffers alternate), divide by 64 and subtract
+//                 the code sum (weights are fed as 64 (w + 1)), rescale, store bf16
 //
 // Work is dealt stream-K style: all (row block, column block) pairs in row-major
 // order, cut into equal contiguous ranges, one per CTA, so every SM streams the
