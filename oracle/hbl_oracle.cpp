@@ -201,6 +201,31 @@ int orc_gemm(const int8_t* q, const int8_t* wt, long T, long K, long N, int32_t*
     return bad ? 20 : 0;
 }
 
+// The normalisation in front of the transform ("LN" in Eq. 7; section 2 builds the model from RMS
+// normalisation, no biases): out[t,k] = x[t,k] / sqrt(mean_k x[t,k]^2 + eps_ln) * g[k], computed in
+// fp64 and rounded once to bf16, the type activations are stored in (returned widened to fp32, every
+// value exactly a bf16).  pre (may be null): the fp64 values before that rounding.
+// Reading taken where the paper is silent: RMS normalisation (no mean subtraction), a learned gain
+// vector, eps_ln inside the square root, result in bf16.  Parity unpinned for those choices.
+int orc_rmsnorm_bf16(const float* x, const float* g, long T, long K, float eps_ln, float* out, double* pre) {
+    if (T < 0 || K <= 0 || eps_ln < 0.0f) return 30;
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < T; ++t) {
+        double ss = 0.0;
+        for (long k = 0; k < K; ++k) ss += (double)x[t * K + k] * (double)x[t * K + k];
+        const double rms = std::sqrt(ss / (double)K + (double)eps_ln);
+        for (long k = 0; k < K; ++k) {
+            const double v = rms > 0.0 ? (double)x[t * K + k] / rms * (double)g[k] : 0.0;
+            if (pre) pre[t * K + k] = v;
+            const uint32_t bits = (uint32_t)bf16_from_double(v) << 16;
+            float f;
+            std::memcpy(&f, &bits, 4);
+            out[t * K + k] = f;
+        }
+    }
+    return 0;
+}
+
 // Eq. 1, 5-7, the prefactors: y[t,o] = alpha * s_t * acc[t,o], rounded once to bf16.
 // y_bits: bf16 bit patterns [T,N]; y64 (may be null): the unrounded fp64 values.
 int orc_rescale(const int32_t* acc, const double* s, float alpha, long T, long N,

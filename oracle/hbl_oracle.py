@@ -61,6 +61,20 @@ def weight_quant(W: np.ndarray, eps: float = 1e-5, prec: int = 32):
     return wt, np.float32(alpha.value)
 
 
+def rmsnorm_bf16(x: np.ndarray, g: np.ndarray, eps_ln: float):
+    """The "LN" of Eq. 7 read as RMS normalisation with a gain vector; fp64, one rounding to bf16.
+    Returns (out float32 [T,K] holding bf16 values, pre float64 [T,K] before that rounding)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    T, K = x.shape
+    assert g.shape == (K,)
+    out = np.empty((T, K), dtype=np.float32)
+    pre = np.empty((T, K), dtype=np.float64)
+    _check(lib().orc_rmsnorm_bf16(_p(x, C.c_float), _p(g, C.c_float), C.c_long(T), C.c_long(K), C.c_float(eps_ln),
+                                  _p(out, C.c_float), _p(pre, C.c_double)), "rmsnorm_bf16")
+    return out, pre
+
+
 def hadamard(x: np.ndarray) -> np.ndarray:
     """Eq. 3-4.  fp32 [T,K] -> fp64 [T,K], orthonormal, natural order."""
     x = np.ascontiguousarray(x, dtype=np.float32)

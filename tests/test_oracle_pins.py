@@ -349,3 +349,61 @@ def test_workload_rows_are_reproducible_and_blockwise():
     assert len(wl.outlier_channels(3, 1, 8192, 0.002)) == 16
     w = wl.CONFIG2.w_latent(0, 64)
     assert abs(w.std() - 0.02) < 5e-4
+
+
+# ------------------------------------------------------------------ normalisation in front of the transform
+def test_rmsnorm_hand_values_and_closed_forms():
+    # 3-4-0-0: mean square 25/4, rms 2.5 -> 1.2, 1.6, 0, 0; in bf16 (8 significant bits) 1.203125 and 1.6015625
+    x = np.array([[3, 4, 0, 0], [-3, 4, 0, 0]], np.float32)
+    out, pre = orc.rmsnorm_bf16(x, np.ones(4, np.float32), 0.0)
+    assert np.allclose(pre, [[1.2, 1.6, 0, 0], [-1.2, 1.6, 0, 0]], rtol=0, atol=1e-15)
+    assert np.array_equal(out, np.array([[1.203125, 1.6015625, 0, 0], [-1.203125, 1.6015625, 0, 0]], np.float32))
+    # a constant vector has rms |c|: the output is sign(c) * g, whatever c
+    g = np.array([0.5, -2.0, 1.0, 3.0, 0.25, 1.5, -1.0, 8.0], np.float32)            # all exactly bf16
+    for c in (1.0, -7.0, 1e-3, 4096.0):
+        out, _ = orc.rmsnorm_bf16(np.full((1, 8), c, np.float32), g, 0.0)
+        assert np.array_equal(out[0], np.sign(c) * g)
+    # the gain multiplies element by element, after the division
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((3, 64)).astype(np.float32)
+    _, p1 = orc.rmsnorm_bf16(x, np.ones(64, np.float32), 0.0)
+    g = rng.uniform(0.5, 2.0, 64).astype(np.float32)
+    _, pg = orc.rmsnorm_bf16(x, g, 0.0)
+    assert np.allclose(pg, p1 * g.astype(np.float64), rtol=1e-15, atol=0)
+    # unit mean square before the gain, and no mean subtraction: adding a constant changes the result
+    assert np.allclose((p1 ** 2).mean(axis=1), 1.0, rtol=1e-12)
+    _, ps = orc.rmsnorm_bf16(x + 1.0, np.ones(64, np.float32), 0.0)
+    assert not np.allclose(ps, p1, atol=1e-3)
+
+
+def test_rmsnorm_scale_behaviour_and_eps():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((4, 128)).astype(np.float32)
+    g = rng.uniform(0.5, 2.0, 128).astype(np.float32)
+    o1, p1 = orc.rmsnorm_bf16(x, g, 0.0)
+    o2, p2 = orc.rmsnorm_bf16(8.0 * x, g, 0.0)                                     # power of two: exact in fp64
+    assert np.array_equal(p1, p2) and np.array_equal(o1, o2)
+    # eps sits under the square root beside the mean square: x / sqrt(ms + eps)
+    ms = (x.astype(np.float64) ** 2).mean(axis=1, keepdims=True)
+    _, pe = orc.rmsnorm_bf16(x, np.ones(128, np.float32), 0.25)
+    assert np.allclose(pe, x / np.sqrt(ms + 0.25), rtol=1e-14, atol=0)
+    # an all-zero token stays zero with eps > 0 (0 / sqrt(eps)) and with eps = 0 (defined as zero)
+    z = np.zeros((1, 128), np.float32)
+    assert not orc.rmsnorm_bf16(z, g, 1e-5)[0].any() and not orc.rmsnorm_bf16(z, g, 0.0)[0].any()
+
+
+def test_rmsnorm_rounds_once_to_bf16():
+    import torch
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((8, 256)).astype(np.float32)
+    g = rng.uniform(0.5, 2.0, 256).astype(np.float32)
+    out, pre = orc.rmsnorm_bf16(x, g, 1e-5)
+    # every output is a bf16 value ...
+    assert np.array_equal(out, torch.from_numpy(out).bfloat16().float().numpy())
+    # ... the nearest one to the fp64 value (ties aside, which a random draw does not hit): the two bf16
+    # neighbours of `pre` found with the library's own float -> bf16 conversion lie no closer
+    lo = torch.from_numpy(pre.astype(np.float32)).bfloat16().float().numpy().astype(np.float64)
+    ulp = 2.0 ** (np.floor(np.log2(np.abs(pre))) - 7)
+    err = np.abs(out.astype(np.float64) - pre)
+    assert np.all(err <= ulp / 2 * (1 + 1e-12))
+    assert np.all(err <= np.abs(lo - pre) + 1e-300)
