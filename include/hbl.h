@@ -103,6 +103,18 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim,
                 int bits, int use_hadamard, float eps, void* y,
                 void* workspace, size_t workspace_bytes, int path, void* stream);
 
+/* hbl_forward with the normalisation of Eq. 7 ("X_r = Hadamard(LN(X))") fused in front of the transform.
+ * The paper does not spell LN out; section 2 builds the model from RMS normalisation without biases, so
+ * LN is taken as  x' = x / sqrt(mean_k x^2 + norm_eps) * gain[k],  computed in fp32 and rounded once to
+ * bf16 (the type activations are handed on in), and x' is what Eq. 3-7 then see.
+ *   x         device, bf16 [tokens, in_dim];  in_dim 2048, 4096, 8192 or 16384 (HBL_ERR_SHAPE otherwise)
+ *   gain      device, fp32 [in_dim], 16-byte aligned, caller-owned
+ *   norm_eps  >= 0 (HBL_ERR_EPS otherwise); the transform is always on
+ * Everything else as hbl_forward. */
+int hbl_forward_norm(const void* x, const float* gain, float norm_eps, int tokens, int in_dim,
+                     const void* W_packed, const float* alpha, int out_dim, int bits, float eps, void* y,
+                     void* workspace, size_t workspace_bytes, int path, void* stream);
+
 /* The seven projections of a LLaMA-like decoder block (section 2): q, k, v and
  * up, gate are plain BitLinear layers (no transform) that share one quantized
  * input each; o and down are H-BitLinear layers (Hadamard on).  Every input is
@@ -167,6 +179,12 @@ int hbl_hadamard_f32(const void* x, int x_dtype, int tokens, int in_dim, float* 
  *   in_dim   2048, 4096, 8192 or 16384 (HBL_ERR_NOT_POW2 / HBL_ERR_SHAPE otherwise); tokens >= 0.
  * Asynchronous on `stream`; returns a status code, allocates nothing. */
 int hbl_hadamard_bf16(const void* g, int tokens, int in_dim, void* out, void* stream);
+
+/* The activation side of hbl_forward_norm alone: normalise, transform, quantize.  With xr_out != NULL
+ * nothing is quantized and xr_out[T,K] fp32 receives H_m x' instead (the other outputs may then be NULL). */
+int hbl_norm_quantize_act(const void* x, const float* gain, float norm_eps, int tokens, int in_dim, int bits,
+                          float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out, float* xr_out,
+                          void* stream);
 
 /* Eq. 3-6: transform (optional), per-token statistic, quantize.  codes_out: int8
  * [T,K], one code per byte; scale_out: fp32 [T] (s_t); codesum_out: int32 [T],

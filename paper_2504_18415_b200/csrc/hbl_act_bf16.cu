@@ -60,6 +60,11 @@ __device__ __forceinline__ f32x2_t fma2(f32x2_t a, f32x2_t b, f32x2_t c) {
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
   return r;
 }
+__device__ __forceinline__ f32x2_t mul2(f32x2_t a, f32x2_t b) {
+  f32x2_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
 __device__ __forceinline__ float fma_sat(float a, float b, float c) {
   float r;
   asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -133,11 +138,14 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int group, in
   return v;
 }
 
-template <int M, int BITS>
+// NORM: the token is RMS-normalised and multiplied by a gain vector first ("LN" of Eq. 7):
+// x' = bf16(x * rsqrt(mean x^2 + norm_eps) * gain), and x' is what the transform sees.
+template <int M, int BITS, bool NORM = false>
 __global__ void __launch_bounds__(Geometry<M>::THREADS, 768 / Geometry<M>::THREADS)
 fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
                        float* __restrict__ scale, int32_t* __restrict__ codesum, float* __restrict__ xr_out,
-                       int32_t* __restrict__ zero_fill, size_t zero_words) {
+                       int32_t* __restrict__ zero_fill, size_t zero_words, const float* __restrict__ gain,
+                       float norm_eps) {
   using G = Geometry<M>;
   constexpr int K = G::K, NT = G::NT, THREADS = G::THREADS, TPC = G::TPC, R = G::R, C = G::C, RUN = G::RUN;
   extern __shared__ __align__(16) float smem[];
@@ -188,6 +196,45 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
 #pragma unroll
     for (int c = 0; c < 8; ++c)
       raw[c] = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)c << (M - 3))));
+    if constexpr (NORM) {
+      // mean square of the token in fp32 (64 values per thread, then the group), one reciprocal
+      // square root, then (x * rstd) * gain rounded once to bf16 -- the transform's exact +-1
+      // products need bf16 inputs, and bf16 is the type a model hands activations on in.
+      // packed fp32 pairs throughout: a bf16 pair widens with one shift and one mask, and the squares,
+      // the two multiplications and the rounding back to a bf16 pair are one instruction per pair each
+      f32x2_t ss2 = pack2(0.f, 0.f);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const f32x2_t v2 = pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+          ss2 = fma2(v2, v2, ss2);
+        }
+      }
+      float ss_lo, ss_hi;
+      unpack2(ss2, ss_lo, ss_hi);
+      const float ss = group_reduce<NT, false>(ss_lo + ss_hi, red_f, group, lane, warp_cta);
+      const float rstd = __frcp_rn(__fsqrt_rn(__fmaf_rn(ss, 1.0f / (float)K, norm_eps)));
+      const f32x2_t rstd2 = pack2(rstd, rstd);
+      const float* gp = gain + (warp << 8) + (lane << 3);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float4 g0 = __ldg(reinterpret_cast<const float4*>(gp + ((size_t)c << (M - 3))));
+        const float4 g1 = __ldg(reinterpret_cast<const float4*>(gp + ((size_t)c << (M - 3)) + 4));
+        const f32x2_t g2[4] = {pack2(g0.x, g0.y), pack2(g0.z, g0.w), pack2(g1.x, g1.y), pack2(g1.z, g1.w)};
+        uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const f32x2_t v2 = pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+          float lo, hi;
+          unpack2(mul2(mul2(v2, rstd2), g2[i]), lo, hi);      // (x * rstd) * gain, each product rounded to fp32
+          const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+          w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        raw[c] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
       // A fragment: (x: m 0,1) rows g, k3 = 0; (z: m 4,5) rows g+8; (y: m 2,3) k3 = 1; (w: m 6,7) both
@@ -439,12 +486,12 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   grid_dependency_wait();   // chain: this kernel is complete only when the one before it is
 }
 
-template <int M, int BITS>
+template <int M, int BITS, bool NORM = false>
 int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
-               int32_t* zf, size_t zw, cudaStream_t s) {
+               int32_t* zf, size_t zw, cudaStream_t s, const float* gain = nullptr, float norm_eps = 0.f) {
   using G = Geometry<M>;
   const size_t smem = sizeof(float) * G::TPC * G::K;
-  auto kern = fwht_quant_bf16_kernel<M, BITS>;
+  auto kern = fwht_quant_bf16_kernel<M, BITS, NORM>;
   if (smem > 48 * 1024) {
     static bool done = false;   // idempotent attribute; a race only repeats the call
     if (!done) {
@@ -455,7 +502,7 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
   const int grid = (T + G::TPC - 1) / G::TPC;
   profile_before(KERNEL_ACT, s);
   HBL_CUDA_OK(launch_dependent(kern, dim3(grid), dim3(G::THREADS), smem, s, static_cast<const __nv_bfloat16*>(x), T, eps,
-                               codes, scale, codesum, xr_out, zf, zw));
+                               codes, scale, codesum, xr_out, zf, zw, gain, norm_eps));
   profile_after(KERNEL_ACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -463,6 +510,20 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
 }
 
 }  // namespace
+
+int launch_norm_act_quant_bf16(const void* x, const float* gain, float norm_eps, int T, int K, int bits, float eps,
+                               int8_t* codes, float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill,
+                               size_t zero_fill_words, cudaStream_t s) {
+#define HBL_CASE(MM)                                                                                              \
+  case (1 << MM):                                                                                                 \
+    return bits == 8 ? launch_one<MM, 8, true>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps) \
+                     : launch_one<MM, 4, true>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps);
+  switch (K) {
+    HBL_CASE(11) HBL_CASE(12) HBL_CASE(13) HBL_CASE(14)
+    default: return HBL_ERR_SHAPE;
+  }
+#undef HBL_CASE
+}
 
 int launch_hadamard_bf16(const void* x, int T, int K, void* out, cudaStream_t s) {
   if (T <= 0) return HBL_OK;

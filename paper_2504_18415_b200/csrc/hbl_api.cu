@@ -192,9 +192,25 @@ int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_
                              static_cast<cudaStream_t>(stream));
 }
 
-int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* W_packed,
-                const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y,
-                void* workspace, size_t workspace_bytes, int path, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// Requirements of the fused normalisation: bf16 input, the transform on, a width the bf16 kernel has.
+int check_norm_args(int x_dtype, int in_dim, const float* gain, float norm_eps, int tokens) {
+  if (x_dtype != HBL_BF16) return HBL_ERR_FORMAT;
+  if (!is_pow2(in_dim)) return HBL_ERR_NOT_POW2;
+  if (!act_quant_bf16_supported(in_dim)) return HBL_ERR_SHAPE;
+  if (!(norm_eps >= 0.0f) || !isfinite(norm_eps)) return HBL_ERR_EPS;
+  if (tokens > 0 && !gain) return HBL_ERR_NULL;
+  if (!aligned(gain, 16)) return HBL_ERR_ALIGN;
+  return HBL_OK;
+}
+
+// hbl_forward and hbl_forward_norm (gain != nullptr: normalise first).
+int forward_impl(const void* x, int x_dtype, const float* gain, float norm_eps, int tokens, int in_dim,
+                 const void* W_packed, const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y,
+                 void* workspace, size_t workspace_bytes, int path, void* stream) {
   int rc = check_dims(tokens, in_dim, out_dim);
   if (rc != HBL_OK) return rc;
   rc = check_quant_args(x_dtype, in_dim, bits, use_hadamard, eps);
@@ -227,10 +243,11 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
     if (rc != HBL_OK) return rc;
     HBL_CUDA_OK(cudaEventRecord(sp->unpacked[0], sp->side));
   }
-  rc = launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale,
-                        stream_path ? codesum : nullptr /* only the streaming kernel needs the code sums */, nullptr,
-                        stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
-                        stream_path ? w.zero_words : 0, s);
+  int32_t* zf = stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr;
+  const size_t zw = stream_path ? w.zero_words : 0;
+  int32_t* cs = stream_path ? codesum : nullptr;             // only the streaming kernel needs the code sums
+  rc = gain ? launch_norm_act_quant_bf16(x, gain, norm_eps, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s)
+            : launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale, cs, nullptr, zf, zw, s);
   if (rc != HBL_OK) {
     if (sp != nullptr) cudaStreamWaitEvent(s, sp->unpacked[0], 0);   // join before reporting the error
     return rc;
@@ -241,6 +258,47 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* 
                               reinterpret_cast<int*>(ws + w.counters), s);
   HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[0], 0));
   return launch_gemm_tensor(codes, scale, tokens, in_dim, w_i8, out_dim, alpha, static_cast<__nv_bfloat16*>(y), nullptr, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* W_packed,
+                const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y,
+                void* workspace, size_t workspace_bytes, int path, void* stream) {
+  return forward_impl(x, x_dtype, nullptr, 0.f, tokens, in_dim, W_packed, alpha, out_dim, bits, use_hadamard, eps, y,
+                      workspace, workspace_bytes, path, stream);
+}
+
+int hbl_forward_norm(const void* x, const float* gain, float norm_eps, int tokens, int in_dim, const void* W_packed,
+                     const float* alpha, int out_dim, int bits, float eps, void* y, void* workspace,
+                     size_t workspace_bytes, int path, void* stream) {
+  const int rc = check_norm_args(HBL_BF16, in_dim, gain, norm_eps, tokens);
+  if (rc != HBL_OK) return rc;
+  return forward_impl(x, HBL_BF16, gain, norm_eps, tokens, in_dim, W_packed, alpha, out_dim, bits, 1, eps, y, workspace,
+                      workspace_bytes, path, stream);
+}
+
+int hbl_norm_quantize_act(const void* x, const float* gain, float norm_eps, int tokens, int in_dim, int bits, float eps,
+                          int8_t* codes_out, float* scale_out, int32_t* codesum_out, float* xr_out, void* stream) {
+  int rc = check_dims(tokens, in_dim, 16);
+  if (rc != HBL_OK) return rc;
+  rc = check_quant_args(HBL_BF16, in_dim, bits, 1, eps);
+  if (rc != HBL_OK) return rc;
+  rc = check_norm_args(HBL_BF16, in_dim, gain, norm_eps, tokens);
+  if (rc != HBL_OK) return rc;
+  if (tokens == 0) return HBL_OK;
+  if (!x) return HBL_ERR_NULL;
+  if (!aligned(x, 16)) return HBL_ERR_ALIGN;
+  if (xr_out == nullptr) {
+    if (!codes_out || !scale_out) return HBL_ERR_NULL;
+    if (!aligned(codes_out, 16)) return HBL_ERR_ALIGN;
+  } else if (!aligned(xr_out, 16)) {
+    return HBL_ERR_ALIGN;
+  }
+  return launch_norm_act_quant_bf16(x, gain, norm_eps, tokens, in_dim, bits, eps, codes_out, scale_out, codesum_out,
+                                    xr_out, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
 // ---- decoder block: four quantizations, seven projections -------------------------------

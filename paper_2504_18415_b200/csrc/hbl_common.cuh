@@ -67,6 +67,10 @@ bool act_quant_bf16_supported(int K);
 int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
                           int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
                           cudaStream_t s);
+// The same with the token RMS-normalised and multiplied by gain[K] (fp32, device) first ("LN" of Eq. 7).
+int launch_norm_act_quant_bf16(const void* x, const float* gain, float norm_eps, int T, int K, int bits, float eps,
+                               int8_t* codes, float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill,
+                               size_t zero_fill_words, cudaStream_t s);
 // The transform alone, bf16 in and out (Eq. 8: the backward pass applies it to the gradient); K as above.
 int launch_hadamard_bf16(const void* x, int T, int K, void* out, cudaStream_t s);
 // Weight side: Eq. 1-2 and the 2-bit format.

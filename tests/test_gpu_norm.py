@@ -1,0 +1,101 @@
+"""GPU parity of the normalisation fused in front of the transform ("LN" of Eq. 7) vs the oracle.
+
+The oracle normalises in fp64 and rounds once to bf16; the kernel normalises in fp32 and rounds once to
+bf16.  Where the exact value lies next to a bf16 rounding boundary the two may land on neighbouring bf16
+values; such an element moves every transformed output of its token by at most 2^-8 |x'| / sqrt(K).  The
+tests bound how often that happens through what it does downstream:
+  * transformed values: |dx_r| <= 1e-4 max_k |x_r| (1e-5 for the fp32 butterflies plus the moved inputs);
+  * codes: as for the plain quantizer (+-1, next to a rounding boundary), with a budget of 1e-3 of them;
+  * layer outputs: the usual 1e-2 max(|y|, row rms)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hbl_oracle as orc
+from paper_2504_18415_b200 import hbl, workloads as wl
+from parity_utils import EPS, check_y, to_dev
+
+pytestmark = pytest.mark.gpu
+NORM_EPS = 1e-5
+
+
+def gain_vector(K, seed):
+    rng = np.random.default_rng(seed)
+    return rng.uniform(0.25, 2.0, K).astype(np.float32)
+
+
+@pytest.mark.parametrize("K", [2048, 4096, 8192, 16384])
+def test_norm_transform_matches_oracle(K):
+    T = 37 if K <= 8192 else 9
+    x = wl.rows("ffn_mid" if K >= 8192 else "attn_out", 500 + K, 1, K, 0, T, "bf16")
+    g = gain_vector(K, K)
+    xn, _ = orc.rmsnorm_bf16(x, g, NORM_EPS)
+    want = orc.hadamard(xn)
+    got = hbl.hbl_norm_quantize_act(to_dev(x, "bf16"), torch.from_numpy(g).cuda(), NORM_EPS, 4, EPS, export_xr=True)
+    got = got.cpu().numpy().astype(np.float64)
+    tol = 1e-4 * np.abs(want).max(axis=1, keepdims=True)
+    assert np.all(np.abs(got - want) <= tol), float((np.abs(got - want) / tol).max())
+
+
+def test_norm_special_cases():
+    K = 4096
+    g = gain_vector(K, 3)
+    gd = torch.from_numpy(g).cuda()
+    # a constant token normalises to the gain vector (exactly, for a gain that is bf16-exact)
+    gb = torch.from_numpy(g).bfloat16().float()
+    x = np.full((2, K), 3.0, np.float32); x[1] = -0.5
+    xr = hbl.hbl_norm_quantize_act(to_dev(x, "bf16"), gb.cuda(), 0.0, 4, EPS, export_xr=True).cpu().numpy()
+    want = orc.hadamard(np.stack([gb.numpy(), -gb.numpy()]))
+    assert np.all(np.abs(xr - want) <= 1e-5 * np.abs(want).max(axis=1, keepdims=True))
+    # scaling a token by a power of two changes nothing when norm_eps is zero
+    y = wl.rows("gauss", 9, 1, K, 0, 6, "bf16")
+    a = hbl.hbl_norm_quantize_act(to_dev(y, "bf16"), gd, 0.0, 4, EPS)
+    b = hbl.hbl_norm_quantize_act(to_dev(4 * y, "bf16"), gd, 0.0, 4, EPS)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    # an all-zero token gives zero codes
+    z = torch.zeros((3, K), dtype=torch.bfloat16, device="cuda")
+    codes, scale, csum = hbl.hbl_norm_quantize_act(z, gd, NORM_EPS, 8, EPS)
+    assert not codes.any() and not csum.any() and hbl.hbl_check_status() == 0
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("K", [2048, 8192])
+def test_norm_quantize_matches_oracle(K, bits):
+    T = 41
+    x = wl.rows("attn_out", 700 + K + bits, 1, K, 0, T, "bf16")
+    g = gain_vector(K, K + 1)
+    xn, _ = orc.rmsnorm_bf16(x, g, NORM_EPS)
+    q, v, s, st = orc.act_quant(orc.hadamard(xn), bits, EPS, 32)
+    codes, scale, csum = hbl.hbl_norm_quantize_act(to_dev(x, "bf16"), torch.from_numpy(g).cuda(), NORM_EPS, bits, EPS)
+    cg = codes.cpu().numpy()
+    diff = cg.astype(np.int32) - q.astype(np.int32)
+    bad = np.nonzero(diff)
+    assert len(bad[0]) <= 1e-3 * q.size, f"{len(bad[0])} of {q.size} codes differ"
+    if len(bad[0]):
+        assert np.all(np.abs(diff[bad]) == 1)
+        b = q[bad].astype(np.float64) + 0.5 * diff[bad]
+        # a moved bf16 input shifts the pre-rounding value v by up to 2^-8 |x'| sqrt(7)/(beta sqrt(K)) ~ 1e-4
+        assert np.all(np.abs(v[bad] - b) <= 2e-3 * np.maximum(1.0, np.abs(b)))
+    assert np.allclose(scale.cpu().numpy(), s, rtol=2e-4, atol=0)
+    assert np.array_equal(csum.cpu().numpy(), cg.astype(np.int64).sum(1))
+
+
+@pytest.mark.parametrize("T", [5, 16, 300])
+def test_forward_norm_matches_oracle(T):
+    K, N = 2048, 784
+    x = wl.rows("attn_out", 900 + T, 1, K, 0, T, "bf16")
+    W = wl.rows("latent", 900 + T, 2, K, 0, N, "f32")
+    g = gain_vector(K, T)
+    packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), EPS)
+    y = hbl.hbl_forward_norm(to_dev(x, "bf16"), torch.from_numpy(g).cuda(), NORM_EPS, packed, alpha, N, 4, EPS)
+    assert hbl.hbl_check_status() == 0
+    xn, _ = orc.rmsnorm_bf16(x, g, NORM_EPS)
+    wt, al = orc.weight_quant(W, EPS, 32)
+    q, v, s, st = orc.act_quant(orc.hadamard(xn), 4, EPS, 32)
+    _, y64 = orc.rescale(orc.gemm(q, wt), s, al)
+    check_y(y, y64)
+    # and it is the plain layer applied to the normalised activations
+    y2 = hbl.hbl_forward(to_dev(xn, "bf16"), packed, alpha, N, 4, True, EPS)
+    yf, y2f = y.float(), y2.float()
+    rms = y2f.pow(2).mean(1, keepdim=True).sqrt()
+    assert torch.all((yf - y2f).abs() <= 1e-2 * torch.maximum(y2f.abs(), rms))
