@@ -226,6 +226,26 @@ int orc_rmsnorm_bf16(const float* x, const float* g, long T, long K, float eps_l
     return 0;
 }
 
+// The input of W_down in a SwishGLU feed-forward block (section 2 names SwishGLU among the model's
+// components): out[t,k] = SiLU(gate[t,k]) * up[t,k] with SiLU(z) = z / (1 + exp(-z)), computed in fp64
+// and rounded once to bf16 (returned widened to fp32).  pre (may be null): the fp64 values before that
+// rounding.  Reading taken where the paper is silent: which projection passes through SiLU (the one
+// called gate here), and bf16 as the type of the product.  Parity unpinned for those choices.
+int orc_swiglu_bf16(const float* gate, const float* up, long T, long K, float* out, double* pre) {
+    if (T < 0 || K <= 0) return 31;
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < T * K; ++i) {
+        const double z = (double)gate[i];
+        const double v = z / (1.0 + std::exp(-z)) * (double)up[i];
+        if (pre) pre[i] = v;
+        const uint32_t bits = (uint32_t)bf16_from_double(v) << 16;
+        float f;
+        std::memcpy(&f, &bits, 4);
+        out[i] = f;
+    }
+    return 0;
+}
+
 // Eq. 1, 5-7, the prefactors: y[t,o] = alpha * s_t * acc[t,o], rounded once to bf16.
 // y_bits: bf16 bit patterns [T,N]; y64 (may be null): the unrounded fp64 values.
 int orc_rescale(const int32_t* acc, const double* s, float alpha, long T, long N,

@@ -75,6 +75,19 @@ def rmsnorm_bf16(x: np.ndarray, g: np.ndarray, eps_ln: float):
     return out, pre
 
 
+def swiglu_bf16(gate: np.ndarray, up: np.ndarray):
+    """SiLU(gate) * up in fp64, one rounding to bf16.  Returns (out float32 holding bf16 values, pre float64)."""
+    gate = np.ascontiguousarray(gate, dtype=np.float32)
+    up = np.ascontiguousarray(up, dtype=np.float32)
+    assert gate.shape == up.shape
+    T, K = gate.shape
+    out = np.empty((T, K), dtype=np.float32)
+    pre = np.empty((T, K), dtype=np.float64)
+    _check(lib().orc_swiglu_bf16(_p(gate, C.c_float), _p(up, C.c_float), C.c_long(T), C.c_long(K),
+                                 _p(out, C.c_float), _p(pre, C.c_double)), "swiglu_bf16")
+    return out, pre
+
+
 def hadamard(x: np.ndarray) -> np.ndarray:
     """Eq. 3-4.  fp32 [T,K] -> fp64 [T,K], orthonormal, natural order."""
     x = np.ascontiguousarray(x, dtype=np.float32)

@@ -407,3 +407,44 @@ def test_rmsnorm_rounds_once_to_bf16():
     err = np.abs(out.astype(np.float64) - pre)
     assert np.all(err <= ulp / 2 * (1 + 1e-12))
     assert np.all(err <= np.abs(lo - pre) + 1e-300)
+
+
+# ------------------------------------------------------------------ SwishGLU in front of W_down
+def test_swiglu_closed_forms():
+    ln3 = math.log(3.0)
+    g = np.array([[0.0, ln3, -ln3, 1.0, -1.0, 40.0, -40.0, 2.5]], np.float32)
+    one = np.ones_like(g)
+    _, pre = orc.swiglu_bf16(g, one)
+    gd = g.astype(np.float64)                                   # the oracle sees the fp32 inputs
+    # sigmoid(ln 3) = 3/4 and sigmoid(-ln 3) = 1/4 (up to ln 3 having been rounded to fp32)
+    assert pre[0, 0] == 0.0
+    assert abs(pre[0, 1] - 0.75 * gd[0, 1]) < 1e-7 and abs(pre[0, 2] - 0.25 * gd[0, 2]) < 1e-7
+    assert abs(pre[0, 3] - 0.7310585786300049) < 1e-15          # 1 / (1 + 1/e)
+    # SiLU(z) - SiLU(-z) = z for every z
+    assert abs((pre[0, 3] - pre[0, 4]) - 1.0) < 1e-15 and abs((pre[0, 1] - pre[0, 2]) - gd[0, 1]) < 1e-15
+    # far out: the identity on the right, zero on the left
+    assert abs(pre[0, 5] - 40.0) < 1e-12 and abs(pre[0, 6]) < 1e-12
+    # the other operand multiplies element by element and is not passed through SiLU
+    u = np.array([[2.0, -1.0, 0.5, 3.0, 0.0, 1.0, 1.0, -4.0]], np.float32)
+    _, pu = orc.swiglu_bf16(g, u)
+    assert np.array_equal(pu, pre * u.astype(np.float64))
+    _, swapped = orc.swiglu_bf16(u, g)
+    assert not np.allclose(swapped, pu)
+
+
+def test_swiglu_derivative_and_single_rounding():
+    import torch
+    # d/dz SiLU(z) = s (1 + z (1 - s)), s = sigmoid(z): check by central differences on exactly representable points
+    z = np.array([[-2.0, -0.5, 0.25, 1.5, 3.0]], np.float32)
+    h = np.float32(2.0 ** -10)
+    _, a = orc.swiglu_bf16(z + h, np.ones_like(z))
+    _, b = orc.swiglu_bf16(z - h, np.ones_like(z))
+    sgm = 1.0 / (1.0 + np.exp(-z.astype(np.float64)))
+    assert np.allclose((a - b) / (2.0 * float(h)), sgm * (1.0 + z * (1.0 - sgm)), rtol=0, atol=1e-6)
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal((4, 256)).astype(np.float32) * 2
+    u = rng.standard_normal((4, 256)).astype(np.float32)
+    out, pre = orc.swiglu_bf16(g, u)
+    assert np.array_equal(out, torch.from_numpy(out).bfloat16().float().numpy())
+    ulp = 2.0 ** (np.floor(np.log2(np.abs(pre))) - 7)
+    assert np.all(np.abs(out.astype(np.float64) - pre) <= ulp / 2 * (1 + 1e-12))
