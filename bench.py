@@ -284,6 +284,37 @@ def norm_quantize_point(K, T, torch, hbl, peaks, iters=None):
     return out
 
 
+def glu_quantize_point(K, T, torch, hbl, peaks, iters=None):
+    """SiLU(gate) * up + transform + INT4 quantizer in one kernel (the activation side of hbl_forward_glu):
+    2 x 2 B read + 1 B written per element, L2-cold."""
+    per_call = 5 * T * K
+    ring = max(2, min(16, -(-RING_BYTES // per_call)))
+    gen = torch.Generator(device="cuda").manual_seed(800 + K)
+    gs = [torch.randn((T, K), device="cuda", generator=gen).bfloat16() for _ in range(ring)]
+    us = [torch.randn((T, K), device="cuda", generator=gen).bfloat16() for _ in range(ring)]
+    codes = torch.empty((T, K), dtype=torch.int8, device="cuda")
+    scale = torch.empty((T,), dtype=torch.float32, device="cuda")
+    L = hbl.lib()
+    state = {"i": 0}
+
+    def call():
+        r = state["i"] % ring
+        state["i"] += 1
+        rc = L.hbl_glu_quantize_act(gs[r].data_ptr(), us[r].data_ptr(), T, K, 4, EPS, codes.data_ptr(), scale.data_ptr(),
+                                    None, None, None)
+        if rc != 0:
+            raise RuntimeError(f"hbl_glu_quantize_act returned {rc}")
+
+    ms = time_loop(call, iters or 30, 3, torch)
+    gbs = per_call / (ms * 1e-3) / 1e9
+    out = {"point": "glu_transform_quantize_int4", "tokens": T, "in": K, "out": K, "bits": 4, "hadamard": True,
+           "ms": round(ms, 5), "tokens_per_s": round(T / (ms * 1e-3), 1), "tops": 0.0, "alg_gbs": round(gbs, 1),
+           "ring": ring, "graph": False, "bound": "hbm", "frac": round(gbs / peaks["hbm_gbs"], 4)}
+    del gs, us
+    torch.cuda.empty_cache()
+    return out
+
+
 def block_point(T, torch, hbl, peaks, iters=None):
     """7B-shaped decoder-block projection sweep point (config 5)."""
     from paper_2504_18415_b200 import workloads as wl
@@ -573,6 +604,8 @@ def main():
                     points.append(backward_transform_point(K_, 16384, torch, hbl, peaks))
                 if want("norm_transform_quantize_int4", 16384):
                     points.append(norm_quantize_point(K_, 16384, torch, hbl, peaks))
+                if want("glu_transform_quantize_int4", 16384):
+                    points.append(glu_quantize_point(K_, 16384, torch, hbl, peaks))
         for T_ in ((1, 4, 16, 64, 256, 1024, 4096, 16384, 65536) if full else (1, 16, 256, 4096)):
             if want("config5_block_7B", T_):
                 points.append(block_point(T_, torch, hbl, peaks))

@@ -115,6 +115,18 @@ int hbl_forward_norm(const void* x, const float* gain, float norm_eps, int token
                      const void* W_packed, const float* alpha, int out_dim, int bits, float eps, void* y,
                      void* workspace, size_t workspace_bytes, int path, void* stream);
 
+/* The down projection of a SwishGLU feed-forward block (section 2 lists SwishGLU among the model's
+ * components and makes W_down an H-BitLinear layer) with the gating product fused in front of the
+ * transform: the layer's input is  x' = SiLU(gate) * up,  SiLU(z) = z / (1 + exp(-z)), computed in fp32
+ * and rounded once to bf16, so the [tokens, in_dim] product never goes to memory.
+ *   gate, up  device, bf16 [tokens, in_dim], 16-byte aligned (the outputs of W_gate and W_up);
+ *             in_dim 2048, 4096, 8192 or 16384 (HBL_ERR_SHAPE otherwise); the transform is always on
+ * Everything else as hbl_forward.  The paper does not say which projection passes through SiLU; here it
+ * is the first argument. */
+int hbl_forward_glu(const void* gate, const void* up, int tokens, int in_dim, const void* W_packed,
+                    const float* alpha, int out_dim, int bits, float eps, void* y, void* workspace,
+                    size_t workspace_bytes, int path, void* stream);
+
 /* The seven projections of a LLaMA-like decoder block (section 2): q, k, v and
  * up, gate are plain BitLinear layers (no transform) that share one quantized
  * input each; o and down are H-BitLinear layers (Hadamard on).  Every input is
@@ -179,6 +191,10 @@ int hbl_hadamard_f32(const void* x, int x_dtype, int tokens, int in_dim, float* 
  *   in_dim   2048, 4096, 8192 or 16384 (HBL_ERR_NOT_POW2 / HBL_ERR_SHAPE otherwise); tokens >= 0.
  * Asynchronous on `stream`; returns a status code, allocates nothing. */
 int hbl_hadamard_bf16(const void* g, int tokens, int in_dim, void* out, void* stream);
+
+/* The activation side of hbl_forward_glu alone: gating product, transform, quantize; xr_out as below. */
+int hbl_glu_quantize_act(const void* gate, const void* up, int tokens, int in_dim, int bits, float eps,
+                         int8_t* codes_out, float* scale_out, int32_t* codesum_out, float* xr_out, void* stream);
 
 /* The activation side of hbl_forward_norm alone: normalise, transform, quantize.  With xr_out != NULL
  * nothing is quantized and xr_out[T,K] fp32 receives H_m x' instead (the other outputs may then be NULL). */

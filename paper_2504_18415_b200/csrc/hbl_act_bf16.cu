@@ -138,13 +138,18 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int group, in
   return v;
 }
 
-// NORM: the token is RMS-normalised and multiplied by a gain vector first ("LN" of Eq. 7):
-// x' = bf16(x * rsqrt(mean x^2 + norm_eps) * gain), and x' is what the transform sees.
-template <int M, int BITS, bool NORM = false>
+// What happens to the token before the transform sees it:
+//   PRE_NONE  nothing;
+//   PRE_NORM  RMS normalisation and a gain vector ("LN" of Eq. 7): x' = bf16(x * rsqrt(mean x^2 + norm_eps) * gain),
+//             aux = gain, fp32 [K];
+//   PRE_GLU   the SwishGLU product that feeds W_down: x' = bf16(SiLU(x) * aux), aux = the other projection's
+//             output, bf16 [T, K] (x is the one that passes through SiLU).
+enum { PRE_NONE = 0, PRE_NORM = 1, PRE_GLU = 2 };
+template <int M, int BITS, int PRE = PRE_NONE>
 __global__ void __launch_bounds__(Geometry<M>::THREADS, 768 / Geometry<M>::THREADS)
 fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
                        float* __restrict__ scale, int32_t* __restrict__ codesum, float* __restrict__ xr_out,
-                       int32_t* __restrict__ zero_fill, size_t zero_words, const float* __restrict__ gain,
+                       int32_t* __restrict__ zero_fill, size_t zero_words, const void* __restrict__ aux,
                        float norm_eps) {
   using G = Geometry<M>;
   constexpr int K = G::K, NT = G::NT, THREADS = G::THREADS, TPC = G::TPC, R = G::R, C = G::C, RUN = G::RUN;
@@ -196,7 +201,28 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
 #pragma unroll
     for (int c = 0; c < 8; ++c)
       raw[c] = __ldg(reinterpret_cast<const uint4*>(src + ((size_t)c << (M - 3))));
-    if constexpr (NORM) {
+    if constexpr (PRE == PRE_GLU) {
+      // SiLU(z) = z / (1 + exp(-z)) with the fast exponential and the fast division (relative error ~2^-21,
+      // far inside the bf16 rounding that follows); exp(-z) overflows to +inf for very negative z and the
+      // quotient becomes -0.
+      const __nv_bfloat16* src2 = static_cast<const __nv_bfloat16*>(aux) + token * K + (warp << 8) + (lane << 3);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 up = __ldg(reinterpret_cast<const uint4*>(src2 + ((size_t)c << (M - 3))));
+        const uint32_t u[4] = {up.x, up.y, up.z, up.w};
+        uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float z0 = __uint_as_float(w[i] << 16), z1 = __uint_as_float(w[i] & 0xFFFF0000u);
+          const float u0 = __uint_as_float(u[i] << 16), u1 = __uint_as_float(u[i] & 0xFFFF0000u);
+          const float s0 = __fdividef(z0, 1.0f + __expf(-z0)), s1 = __fdividef(z1, 1.0f + __expf(-z1));
+          const __nv_bfloat162 h = __floats2bfloat162_rn(s0 * u0, s1 * u1);
+          w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        raw[c] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+    if constexpr (PRE == PRE_NORM) {
       // mean square of the token in fp32 (64 values per thread, then the group), one reciprocal
       // square root, then (x * rstd) * gain rounded once to bf16 -- the transform's exact +-1
       // products need bf16 inputs, and bf16 is the type a model hands activations on in.
@@ -217,7 +243,7 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
       const float ss = group_reduce<NT, false>(ss_lo + ss_hi, red_f, group, lane, warp_cta);
       const float rstd = __frcp_rn(__fsqrt_rn(__fmaf_rn(ss, 1.0f / (float)K, norm_eps)));
       const f32x2_t rstd2 = pack2(rstd, rstd);
-      const float* gp = gain + (warp << 8) + (lane << 3);
+      const float* gp = static_cast<const float*>(aux) + (warp << 8) + (lane << 3);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const float4 g0 = __ldg(reinterpret_cast<const float4*>(gp + ((size_t)c << (M - 3))));
@@ -486,12 +512,12 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   grid_dependency_wait();   // chain: this kernel is complete only when the one before it is
 }
 
-template <int M, int BITS, bool NORM = false>
+template <int M, int BITS, int PRE = PRE_NONE>
 int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
-               int32_t* zf, size_t zw, cudaStream_t s, const float* gain = nullptr, float norm_eps = 0.f) {
+               int32_t* zf, size_t zw, cudaStream_t s, const void* aux = nullptr, float norm_eps = 0.f) {
   using G = Geometry<M>;
   const size_t smem = sizeof(float) * G::TPC * G::K;
-  auto kern = fwht_quant_bf16_kernel<M, BITS, NORM>;
+  auto kern = fwht_quant_bf16_kernel<M, BITS, PRE>;
   if (smem > 48 * 1024) {
     static bool done = false;   // idempotent attribute; a race only repeats the call
     if (!done) {
@@ -502,7 +528,7 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
   const int grid = (T + G::TPC - 1) / G::TPC;
   profile_before(KERNEL_ACT, s);
   HBL_CUDA_OK(launch_dependent(kern, dim3(grid), dim3(G::THREADS), smem, s, static_cast<const __nv_bfloat16*>(x), T, eps,
-                               codes, scale, codesum, xr_out, zf, zw, gain, norm_eps));
+                               codes, scale, codesum, xr_out, zf, zw, aux, norm_eps));
   profile_after(KERNEL_ACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -516,8 +542,22 @@ int launch_norm_act_quant_bf16(const void* x, const float* gain, float norm_eps,
                                size_t zero_fill_words, cudaStream_t s) {
 #define HBL_CASE(MM)                                                                                              \
   case (1 << MM):                                                                                                 \
-    return bits == 8 ? launch_one<MM, 8, true>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps) \
-                     : launch_one<MM, 4, true>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps);
+    return bits == 8 ? launch_one<MM, 8, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps) \
+                     : launch_one<MM, 4, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps);
+  switch (K) {
+    HBL_CASE(11) HBL_CASE(12) HBL_CASE(13) HBL_CASE(14)
+    default: return HBL_ERR_SHAPE;
+  }
+#undef HBL_CASE
+}
+
+int launch_glu_act_quant_bf16(const void* gate, const void* up, int T, int K, int bits, float eps, int8_t* codes,
+                              float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
+                              cudaStream_t s) {
+#define HBL_CASE(MM)                                                                                              \
+  case (1 << MM):                                                                                                 \
+    return bits == 8 ? launch_one<MM, 8, PRE_GLU>(gate, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, up, 0.f) \
+                     : launch_one<MM, 4, PRE_GLU>(gate, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, up, 0.f);
   switch (K) {
     HBL_CASE(11) HBL_CASE(12) HBL_CASE(13) HBL_CASE(14)
     default: return HBL_ERR_SHAPE;

@@ -71,6 +71,10 @@ int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8
 int launch_norm_act_quant_bf16(const void* x, const float* gain, float norm_eps, int T, int K, int bits, float eps,
                                int8_t* codes, float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill,
                                size_t zero_fill_words, cudaStream_t s);
+// The same with the token replaced by SiLU(gate) * up first (both bf16 [T, K]): the SwishGLU input of W_down.
+int launch_glu_act_quant_bf16(const void* gate, const void* up, int T, int K, int bits, float eps, int8_t* codes,
+                              float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
+                              cudaStream_t s);
 // The transform alone, bf16 in and out (Eq. 8: the backward pass applies it to the gradient); K as above.
 int launch_hadamard_bf16(const void* x, int T, int K, void* out, cudaStream_t s);
 // Weight side: Eq. 1-2 and the 2-bit format.

@@ -25,7 +25,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "hbl_status_string", "hbl_packed_weight_bytes", "hbl_workspace_bytes",
     "hbl_quantize_weights_workspace_bytes", "hbl_quantize_weights", "hbl_forward",
-    "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act",
+    "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_forward_glu", "hbl_glu_quantize_act",
     "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
     "hbl_profile_events", "hbl_gemm_i32_static",
 ]
@@ -73,6 +73,8 @@ def lib() -> C.CDLL:
         L.hbl_hadamard_bf16.argtypes = [vp, i, i, vp, vp]
         L.hbl_forward_norm.argtypes = [vp, vp, f, i, i, vp, vp, i, i, f, vp, vp, sz, i, vp]
         L.hbl_norm_quantize_act.argtypes = [vp, vp, f, i, i, i, f, vp, vp, vp, vp, vp]
+        L.hbl_forward_glu.argtypes = [vp, vp, i, i, vp, vp, i, i, f, vp, vp, sz, i, vp]
+        L.hbl_glu_quantize_act.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp]
         L.hbl_quantize_act.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp]
         L.hbl_gemm_i32.argtypes = [vp, vp, i, i, vp, i, vp, vp, sz, i, vp]
         L.hbl_unpack_weights.argtypes = [vp, i, i, vp, vp]
@@ -85,7 +87,7 @@ def lib() -> C.CDLL:
         L.hbl_profile_events.argtypes = [C.POINTER(vp), C.POINTER(vp), i, i]
         L.hbl_profile_events.restype = C.c_int
         for n in ("hbl_quantize_weights", "hbl_forward", "hbl_block_forward", "hbl_check_status",
-                  "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights"):
+                  "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_forward_glu", "hbl_glu_quantize_act", "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -223,6 +225,36 @@ def hbl_forward_norm(x: torch.Tensor, gain: torch.Tensor, norm_eps: float, W_pac
     _check(lib().hbl_forward_norm(_ptr(x), _ptr(gain), norm_eps, T, K, _ptr(W_packed), _ptr(alpha), out_dim, bits, eps,
                                   _ptr(y), _ptr(workspace), workspace.numel(), path, _stream()), "hbl_forward_norm")
     return y
+
+
+def hbl_forward_glu(gate: torch.Tensor, up: torch.Tensor, W_packed: torch.Tensor, alpha: torch.Tensor, out_dim: int,
+                    bits: int, eps: float = 1e-5, y: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+                    path: int = PATH_AUTO) -> torch.Tensor:
+    """The down projection with SiLU(gate) * up fused in front of the transform (bf16 gate and up)."""
+    T, K = gate.shape
+    if y is None:
+        y = torch.empty((T, out_dim), dtype=torch.bfloat16, device=gate.device)
+    if workspace is None:
+        workspace = new_workspace(hbl_workspace_bytes(T, K, out_dim), gate.device)
+    _check(lib().hbl_forward_glu(_ptr(gate), _ptr(up), T, K, _ptr(W_packed), _ptr(alpha), out_dim, bits, eps, _ptr(y),
+                                 _ptr(workspace), workspace.numel(), path, _stream()), "hbl_forward_glu")
+    return y
+
+
+def hbl_glu_quantize_act(gate: torch.Tensor, up: torch.Tensor, bits: int, eps: float = 1e-5, export_xr: bool = False):
+    """Gating product, transform, quantize.  Returns (codes, scale, codesum), or the fp32 H x' when export_xr."""
+    T, K = gate.shape
+    if export_xr:
+        xr = torch.empty((T, K), dtype=torch.float32, device=gate.device)
+        _check(lib().hbl_glu_quantize_act(_ptr(gate), _ptr(up), T, K, bits, eps, None, None, None, _ptr(xr), _stream()),
+               "hbl_glu_quantize_act")
+        return xr
+    codes = torch.empty((T, K), dtype=torch.int8, device=gate.device)
+    scale = torch.empty((T,), dtype=torch.float32, device=gate.device)
+    csum = torch.empty((T,), dtype=torch.int32, device=gate.device)
+    _check(lib().hbl_glu_quantize_act(_ptr(gate), _ptr(up), T, K, bits, eps, _ptr(codes), _ptr(scale), _ptr(csum), None,
+                                      _stream()), "hbl_glu_quantize_act")
+    return codes, scale, csum
 
 
 def hbl_norm_quantize_act(x: torch.Tensor, gain: torch.Tensor, norm_eps: float, bits: int, eps: float = 1e-5,

@@ -71,6 +71,9 @@ def test_argument_errors_come_before_any_launch(L):
     assert L.hbl_norm_quantize_act(p, n, 1e-5, 4, 4096, 4, 1e-5, p, p, p, n, n) == 1      # no gain
     assert L.hbl_norm_quantize_act(p, p, 1e-5, 4, 1024, 4, 1e-5, p, p, p, n, n) == 2      # width without a fused kernel
     assert L.hbl_forward_norm(p, p, 1e-5, 4, 384, p, p, 512, 4, 1e-5, p, p, 1 << 30, 0, n) == 3
+    assert L.hbl_glu_quantize_act(p, n, 4, 4096, 4, 1e-5, p, p, p, n, n) == 1             # no `up`
+    assert L.hbl_glu_quantize_act(p, p, 4, 1024, 4, 1e-5, p, p, p, n, n) == 2
+    assert L.hbl_forward_glu(p, p, 4, 384, p, p, 512, 4, 1e-5, p, p, 1 << 30, 0, n) == 3
     assert L.hbl_hadamard_bf16(p, 4, 384, p, n) == 3             # not a power of two
     assert L.hbl_hadamard_bf16(p, 4, 1024, p, n) == 2            # outside 2048..16384
     assert L.hbl_hadamard_bf16(n, 4, 4096, p, n) == 1

@@ -5,15 +5,16 @@ bf16.  Where the exact value lies next to a bf16 rounding boundary the two may l
 values; such an element moves every transformed output of its token by at most 2^-8 |x'| / sqrt(K).  The
 tests bound how often that happens through what it does downstream:
   * transformed values: |dx_r| <= 1e-4 max_k |x_r| (1e-5 for the fp32 butterflies plus the moved inputs);
-  * codes: as for the plain quantizer (+-1, next to a rounding boundary), with a budget of 1e-3 of them;
-  * layer outputs: the usual 1e-2 max(|y|, row rms)."""
+  * everything after the rounding: the kernel's own roundings are recovered and checked one by one
+    (parity_utils.reconcile_bf16_inputs) and the oracle continues from them, so codes, scales and outputs
+    meet the plain layer's bars."""
 import numpy as np
 import pytest
 import torch
 
 from oracle import hbl_oracle as orc
 from paper_2504_18415_b200 import hbl, workloads as wl
-from parity_utils import EPS, check_y, to_dev
+from parity_utils import EPS, check_codes, check_y, reconcile_bf16_inputs, to_dev
 
 pytestmark = pytest.mark.gpu
 NORM_EPS = 1e-5
@@ -64,19 +65,17 @@ def test_norm_quantize_matches_oracle(K, bits):
     T = 41
     x = wl.rows("attn_out", 700 + K + bits, 1, K, 0, T, "bf16")
     g = gain_vector(K, K + 1)
-    xn, _ = orc.rmsnorm_bf16(x, g, NORM_EPS)
-    q, v, s, st = orc.act_quant(orc.hadamard(xn), bits, EPS, 32)
-    codes, scale, csum = hbl.hbl_norm_quantize_act(to_dev(x, "bf16"), torch.from_numpy(g).cuda(), NORM_EPS, bits, EPS)
+    xd, gd = to_dev(x, "bf16"), torch.from_numpy(g).cuda()
+    xn, pre = orc.rmsnorm_bf16(x, g, NORM_EPS)
+    xk, n_moved = reconcile_bf16_inputs(hbl.hbl_norm_quantize_act(xd, gd, NORM_EPS, bits, EPS, export_xr=True), xn, pre)
+    assert n_moved <= 1e-3 * xn.size
+    q, v, s, st = orc.act_quant(orc.hadamard(xk), bits, EPS, 32)
+    codes, scale, csum = hbl.hbl_norm_quantize_act(xd, gd, NORM_EPS, bits, EPS)
     cg = codes.cpu().numpy()
-    diff = cg.astype(np.int32) - q.astype(np.int32)
-    bad = np.nonzero(diff)
-    assert len(bad[0]) <= 1e-3 * q.size, f"{len(bad[0])} of {q.size} codes differ"
-    if len(bad[0]):
-        assert np.all(np.abs(diff[bad]) == 1)
-        b = q[bad].astype(np.float64) + 0.5 * diff[bad]
-        # a moved bf16 input shifts the pre-rounding value v by up to 2^-8 |x'| sqrt(7)/(beta sqrt(K)) ~ 1e-4
-        assert np.all(np.abs(v[bad] - b) <= 2e-3 * np.maximum(1.0, np.abs(b)))
-    assert np.allclose(scale.cpu().numpy(), s, rtol=2e-4, atol=0)
+    # elements too small to recover from the export may have been rounded the other way unnoticed: each moves
+    # the pre-rounding values by ~1e-5, on top of the fp32 butterflies' own error
+    check_codes(cg, q, v, near=4e-5)
+    assert np.allclose(scale.cpu().numpy(), s, rtol=5e-5, atol=0)      # fp32 butterflies vs fp64 on heavy-tailed rows
     assert np.array_equal(csum.cpu().numpy(), cg.astype(np.int64).sum(1))
 
 
@@ -89,13 +88,17 @@ def test_forward_norm_matches_oracle(T):
     packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), EPS)
     y = hbl.hbl_forward_norm(to_dev(x, "bf16"), torch.from_numpy(g).cuda(), NORM_EPS, packed, alpha, N, 4, EPS)
     assert hbl.hbl_check_status() == 0
-    xn, _ = orc.rmsnorm_bf16(x, g, NORM_EPS)
+    xd, gd = to_dev(x, "bf16"), torch.from_numpy(g).cuda()
+    xn, pre = orc.rmsnorm_bf16(x, g, NORM_EPS)
+    xk, n_moved = reconcile_bf16_inputs(hbl.hbl_norm_quantize_act(xd, gd, NORM_EPS, 4, EPS, export_xr=True), xn, pre)
+    assert n_moved <= 1e-3 * xn.size
     wt, al = orc.weight_quant(W, EPS, 32)
-    q, v, s, st = orc.act_quant(orc.hadamard(xn), 4, EPS, 32)
+    q, v, s, st = orc.act_quant(orc.hadamard(xk), 4, EPS, 32)
     _, y64 = orc.rescale(orc.gemm(q, wt), s, al)
     check_y(y, y64)
-    # and it is the plain layer applied to the normalised activations
-    y2 = hbl.hbl_forward(to_dev(xn, "bf16"), packed, alpha, N, 4, True, EPS)
-    yf, y2f = y.float(), y2.float()
-    rms = y2f.pow(2).mean(1, keepdim=True).sqrt()
-    assert torch.all((yf - y2f).abs() <= 1e-2 * torch.maximum(y2f.abs(), rms))
+    # the plain layer applied to the normalised activations (with the kernel's roundings) gives the same values
+    # (up to roundings of elements too small to recover from the export, which can move a code or two)
+    y2 = hbl.hbl_forward(to_dev(xk, "bf16"), packed, alpha, N, 4, True, EPS).float()
+    rms = y2.pow(2).mean(1, keepdim=True).sqrt()
+    assert torch.all((y.float() - y2).abs() <= 1e-2 * torch.maximum(y2.abs(), rms))
+    assert (y.float() != y2).float().mean() <= 1e-2
