@@ -84,6 +84,19 @@ int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_
                          void* W_packed, float* alpha, void* workspace, size_t workspace_bytes,
                          void* stream);
 
+/* The "weight and activation rotation" variant of the ablation (section 4.2, Table 5): the transform is
+ * applied to the weights as well, W' = W H_m, and W' is ternarised in place of W; with use_hadamard = 1
+ * the layer then computes Q_w(W H) Q(H x), and (W H)(H x) = W x before quantization.  The paper gives no
+ * formula beyond that sentence; here each weight row is transformed (orthonormal, natural order, fp32,
+ * H_m is symmetric) and Eq. 1-2 are applied to the fp32 result.  in_dim must be a power of two.
+ * Workspace: hbl_quantize_weights_rotated_workspace_bytes (it holds the fp32 copy of W H), 256-byte
+ * aligned.  Everything else as hbl_quantize_weights; the result equals hbl_hadamard_f32 on the rows
+ * followed by hbl_quantize_weights. */
+size_t hbl_quantize_weights_rotated_workspace_bytes(int out_dim, int in_dim);
+int hbl_quantize_weights_rotated(const void* W_latent, int w_dtype, int out_dim, int in_dim, float eps,
+                                 void* W_packed, float* alpha, void* workspace, size_t workspace_bytes,
+                                 void* stream);
+
 /* Eq. 3-7: the layer's forward pass for `tokens` tokens.
  *   x         [tokens, in_dim] fp32 or bf16
  *   W_packed  from hbl_quantize_weights;  alpha: device pointer to its scale

@@ -192,6 +192,35 @@ int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_
                              static_cast<cudaStream_t>(stream));
 }
 
+size_t hbl_quantize_weights_rotated_workspace_bytes(int out_dim, int in_dim) {
+  const size_t base = hbl_quantize_weights_workspace_bytes(out_dim, in_dim);
+  if (base == 0) return 0;
+  return align_up(base, 256) + sizeof(float) * (size_t)out_dim * in_dim;
+}
+
+int hbl_quantize_weights_rotated(const void* W_latent, int w_dtype, int out_dim, int in_dim, float eps,
+                                 void* W_packed, float* alpha, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+  if (!W_latent || !W_packed || !alpha || !workspace) return HBL_ERR_NULL;
+  int rc = check_dims(0, in_dim, out_dim);
+  if (rc != HBL_OK) return rc;
+  if (w_dtype != HBL_F32 && w_dtype != HBL_BF16) return HBL_ERR_FORMAT;
+  if (!is_pow2(in_dim)) return HBL_ERR_NOT_POW2;
+  if (!(eps > 0.0f) || !isfinite(eps)) return HBL_ERR_EPS;
+  if (!aligned(W_latent, 16) || !aligned(W_packed, 16) || !aligned(alpha, 4) || !aligned(workspace, 256))
+    return HBL_ERR_ALIGN;
+  if (workspace_bytes < hbl_quantize_weights_rotated_workspace_bytes(out_dim, in_dim)) return HBL_ERR_WORKSPACE;
+  const size_t base = align_up(hbl_quantize_weights_workspace_bytes(out_dim, in_dim), 256);
+  float* rotated = reinterpret_cast<float*>(static_cast<char*>(workspace) + base);
+  // rows of W H are the transforms of the rows of W (H is symmetric): the activation kernel's transform-only
+  // mode, with the weight rows in the place of tokens, then Eq. 1-2 on the result
+  rc = launch_act_quant(W_latent, w_dtype, out_dim, in_dim, 4, 1, 1.0f, nullptr, nullptr, nullptr, rotated, nullptr, 0,
+                        static_cast<cudaStream_t>(stream));
+  if (rc != HBL_OK) return rc;
+  return launch_weight_quant(rotated, HBL_F32, out_dim, in_dim, eps, W_packed, alpha, workspace,
+                             static_cast<cudaStream_t>(stream));
+}
+
 }  // extern "C"
 
 namespace {

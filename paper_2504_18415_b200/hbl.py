@@ -25,7 +25,7 @@ STATUS_NAMES = {
 EXPORTS = [
     "hbl_status_string", "hbl_packed_weight_bytes", "hbl_workspace_bytes",
     "hbl_quantize_weights_workspace_bytes", "hbl_quantize_weights", "hbl_forward",
-    "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_forward_glu", "hbl_glu_quantize_act",
+    "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_forward_glu", "hbl_glu_quantize_act", "hbl_quantize_weights_rotated", "hbl_quantize_weights_rotated_workspace_bytes",
     "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
     "hbl_profile_events", "hbl_gemm_i32_static",
 ]
@@ -58,7 +58,8 @@ def lib() -> C.CDLL:
         L = C.CDLL(LIB_PATH)
         L.hbl_status_string.restype = C.c_char_p
         L.hbl_status_string.argtypes = [C.c_int]
-        for n in ("hbl_packed_weight_bytes", "hbl_quantize_weights_workspace_bytes"):
+        for n in ("hbl_packed_weight_bytes", "hbl_quantize_weights_workspace_bytes",
+                  "hbl_quantize_weights_rotated_workspace_bytes"):
             getattr(L, n).restype = C.c_size_t
             getattr(L, n).argtypes = [C.c_int, C.c_int]
         for n in ("hbl_workspace_bytes", "hbl_block_workspace_bytes"):
@@ -66,6 +67,8 @@ def lib() -> C.CDLL:
             getattr(L, n).argtypes = [C.c_int, C.c_int, C.c_int]
         vp, i, f, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
         L.hbl_quantize_weights.argtypes = [vp, i, i, i, f, vp, vp, vp, sz, vp]
+        L.hbl_quantize_weights_rotated.argtypes = [vp, i, i, i, f, vp, vp, vp, sz, vp]
+        L.hbl_quantize_weights_rotated.restype = C.c_int
         L.hbl_forward.argtypes = [vp, i, i, i, vp, vp, i, i, i, f, vp, vp, sz, i, vp]
         L.hbl_block_forward.argtypes = [C.POINTER(hbl_block_t), vp, sz, i, vp]
         L.hbl_check_status.argtypes = [vp]
@@ -149,6 +152,22 @@ def hbl_quantize_weights(W_latent: torch.Tensor, eps: float = 1e-5):
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=W_latent.device)
     _check(lib().hbl_quantize_weights(_ptr(W_latent), _dt(W_latent), N, K, eps, _ptr(packed), _ptr(alpha),
                                       _ptr(ws), ws_bytes, _stream()), "hbl_quantize_weights")
+    return packed, alpha
+
+
+def hbl_quantize_weights_rotated(W_latent: torch.Tensor, eps: float = 1e-5):
+    """Ternarises W H (each row transformed first): the weight-and-activation-rotation variant.  Returns as
+    hbl_quantize_weights."""
+    N, K = W_latent.shape
+    nbytes = hbl_packed_weight_bytes(N, K)
+    if nbytes == 0:
+        raise HblError(2, "hbl_quantize_weights_rotated")
+    packed = torch.empty(nbytes, dtype=torch.uint8, device=W_latent.device)
+    alpha = torch.empty(1, dtype=torch.float32, device=W_latent.device)
+    ws_bytes = int(lib().hbl_quantize_weights_rotated_workspace_bytes(N, K))
+    ws = new_workspace(ws_bytes, W_latent.device)
+    _check(lib().hbl_quantize_weights_rotated(_ptr(W_latent), _dt(W_latent), N, K, eps, _ptr(packed), _ptr(alpha),
+                                              _ptr(ws), ws.numel(), _stream()), "hbl_quantize_weights_rotated")
     return packed, alpha
 
 

@@ -74,6 +74,10 @@ def test_argument_errors_come_before_any_launch(L):
     assert L.hbl_glu_quantize_act(p, n, 4, 4096, 4, 1e-5, p, p, p, n, n) == 1             # no `up`
     assert L.hbl_glu_quantize_act(p, p, 4, 1024, 4, 1e-5, p, p, p, n, n) == 2
     assert L.hbl_forward_glu(p, p, 4, 384, p, p, 512, 4, 1e-5, p, p, 1 << 30, 0, n) == 3
+    qr = L.hbl_quantize_weights_rotated
+    assert qr(p, 0, 512, 384, 1e-5, p, p, p, 1 << 30, n) == 3                                # W H needs in_dim = 2^m
+    assert qr(p, 0, 512, 512, 1e-5, p, p, p, 1 << 16, n) == 6                                # no room for the fp32 copy of W H
+    assert L.hbl_quantize_weights_rotated_workspace_bytes(512, 512) >= 4 * 512 * 512
     assert L.hbl_hadamard_bf16(p, 4, 384, p, n) == 3             # not a power of two
     assert L.hbl_hadamard_bf16(p, 4, 1024, p, n) == 2            # outside 2048..16384
     assert L.hbl_hadamard_bf16(n, 4, 4096, p, n) == 1

@@ -61,3 +61,47 @@ def test_weight_quant_special_values():
     wt, a = orc.weight_quant(W, EPS, 32)
     assert alpha.item() == a
     assert np.array_equal(hbl.hbl_unpack_weights(packed, N, K).cpu().numpy(), wt)
+
+
+@pytest.mark.parametrize("N,K,dtype", [(144, 512, "f32"), (528, 2048, "f32"), (256, 8192, "bf16"), (2048, 4096, "f32")])
+def test_rotated_weight_quant(N, K, dtype):
+    """Weight-and-activation rotation (the ablation's other variant): W H is ternarised instead of W.
+    Two stages, each against the oracle: the transformed rows (fp32 butterflies vs the fp64 transform), then
+    Eq. 1-2 on exactly the fp32 values the kernel produced (bit-exact, as for the plain weights) -- the ternary
+    decision is taken on the same numbers on both sides."""
+    import torch
+    from oracle import hbl_oracle as orc
+    W = wl.rows("latent", 60 + N, 7, K, 0, N, dtype)
+    Wd = torch.from_numpy(W).cuda()
+    if dtype == "bf16":
+        Wd = Wd.bfloat16()
+    packed, alpha = hbl.hbl_quantize_weights_rotated(Wd, EPS)
+    assert hbl.hbl_check_status() == 0
+    Wr = hbl.hbl_hadamard_f32(Wd)
+    want = orc.hadamard(W)
+    assert np.all(np.abs(Wr.cpu().numpy() - want) <= 1e-5 * np.abs(want).max(axis=1, keepdims=True))
+    wt, al = orc.weight_quant(Wr.cpu().numpy(), EPS, 32)
+    assert alpha.item() == al
+    assert np.array_equal(hbl.hbl_unpack_weights(packed, N, K).cpu().numpy(), wt)
+    # the same as the two public steps one after the other
+    p2, a2 = hbl.hbl_quantize_weights(Wr, EPS)
+    assert torch.equal(packed, p2) and torch.equal(alpha, a2)
+
+
+def test_rotated_weights_in_the_layer():
+    """With both sides rotated the layer still approximates W x: (W H)(H x) = W x before quantization."""
+    import torch
+    from oracle import hbl_oracle as orc
+    from parity_utils import check_y, oracle_layer, to_dev
+    N, K, T = 272, 2048, 24
+    W = wl.rows("latent", 71, 7, K, 0, N, "f32")
+    x = wl.rows("attn_out", 71, 1, K, 0, T, "bf16")
+    Wd = torch.from_numpy(W).cuda()
+    packed, alpha = hbl.hbl_quantize_weights_rotated(Wd, EPS)
+    y = hbl.hbl_forward(to_dev(x, "bf16"), packed, alpha, N, 8, True, EPS)
+    o = oracle_layer(x, hbl.hbl_hadamard_f32(Wd).cpu().numpy(), 8, True)      # the oracle's layer on the rotated latents
+    check_y(y, o["y64"])
+    dense = x.astype(np.float64) @ W.astype(np.float64).T
+    yf = y.float().cpu().numpy().astype(np.float64)
+    corr = (yf * dense).sum() / np.sqrt((yf ** 2).sum() * (dense ** 2).sum())
+    assert corr > 0.8                                                          # ternary weights: a coarse but aligned product
