@@ -145,7 +145,10 @@ int hbl_forward_glu(const void* gate, const void* up, int tokens, int in_dim, co
  * input each; o and down are H-BitLinear layers (Hadamard on).  Every input is
  * supplied by the caller; attention, RoPE, SwishGLU and residuals are not part
  * of this call.  alpha7: device array of the seven per-tensor alphas in the
- * order q, k, v, o, up, gate, down. */
+ * order q, k, v, o, up, gate, down.
+ * x_down_in may be NULL: the feed-forward block is then chained inside the call, the down projection
+ * taking SiLU(ygate) * yup (as hbl_forward_glu does) from the two outputs it has just written; ffn must
+ * then be 2048, 4096, 8192 or 16384. */
 typedef struct {
   const void *x_attn_in, *x_o_in, *x_ffn_in, *x_down_in; /* [T,H] [T,H] [T,H] [T,F] */
   const void *Wq, *Wk, *Wv, *Wo, *Wup, *Wgate, *Wdown;    /* packed ternary */

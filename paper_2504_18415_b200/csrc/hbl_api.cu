@@ -410,7 +410,11 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   const void* xs[4] = {b->x_attn_in, b->x_o_in, b->x_ffn_in, b->x_down_in};
   const void* Ws[7] = {b->Wq, b->Wk, b->Wv, b->Wo, b->Wup, b->Wgate, b->Wdown};
   void* ys[7] = {b->yq, b->yk, b->yv, b->yo, b->yup, b->ygate, b->ydown};
-  for (int i = 0; i < 4; ++i) {
+  // x_down_in == NULL: the feed-forward block is chained for real -- the down projection's input is
+  // SiLU(ygate) * yup, formed inside its activation kernel from the two outputs written by this call
+  const bool chain_ffn = (b->x_down_in == nullptr);
+  if (chain_ffn && !act_quant_bf16_supported(F)) return HBL_ERR_SHAPE;
+  for (int i = 0; i < (chain_ffn ? 3 : 4); ++i) {
     if (!xs[i]) return HBL_ERR_NULL;
     if (!aligned(xs[i], 16)) return HBL_ERR_ALIGN;
   }
@@ -436,7 +440,7 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     HBL_CUDA_OK(cudaEventRecord(sp->fork, s));
     HBL_CUDA_OK(cudaStreamWaitEvent(sp->side, sp->fork, 0));
   }
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < (chain_ffn ? 3 : 4); ++i) {
     rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
                           reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
                           stream_path ? reinterpret_cast<int32_t*>(ws + w.codesum[i]) : nullptr, nullptr,
@@ -455,8 +459,20 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     StreamJob jobs[7];
     for (int i = 0; i < 7; ++i)
       jobs[i] = {Ws[i], b->alpha7 + i, static_cast<__nv_bfloat16*>(ys[i]), nullptr, out_dims[i], src[i]};
-    return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, reinterpret_cast<int32_t*>(ws + w.acc[0]),
-                                    reinterpret_cast<int*>(ws + w.counters[0]), s);
+    int32_t* part = reinterpret_cast<int32_t*>(ws + w.acc[0]);
+    int* flags = reinterpret_cast<int*>(ws + w.counters[0]);
+    if (!chain_ffn) return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, part, flags, s);
+    // chained: six projections, then the gating product + quantizer (which also clears the flags again: it
+    // starts only when the first launch has completed), then the down projection
+    rc = launch_gemm_stream_multi(inputs, 3, jobs, 6, T, part, flags, s);
+    if (rc != HBL_OK) return rc;
+    rc = launch_glu_act_quant_bf16(ys[5], ys[4], T, F, b->bits, b->eps, reinterpret_cast<int8_t*>(ws + w.codes[3]),
+                                   reinterpret_cast<float*>(ws + w.scale[3]), reinterpret_cast<int32_t*>(ws + w.codesum[3]),
+                                   nullptr, reinterpret_cast<int32_t*>(ws + w.zero_region), w.zero_words, s);
+    if (rc != HBL_OK) return rc;
+    StreamJob down = jobs[6];
+    down.input = 0;
+    return launch_gemm_stream_multi(&inputs[3], 1, &down, 1, T, part, flags, s);
   }
   // Large batch: tensor i+1 is expanded to int8 on the side stream (two buffers alternate) while tensor i
   // is contracted on the caller's stream.
@@ -469,6 +485,11 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     if (rc != HBL_OK) break;
     HBL_CUDA_OK(cudaEventRecord(sp->unpacked[i], sp->side));
     HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[i], 0));
+    if (chain_ffn && i == 6) {                                // up and gate are complete in stream order
+      rc = launch_glu_act_quant_bf16(ys[5], ys[4], T, F, b->bits, b->eps, reinterpret_cast<int8_t*>(ws + w.codes[3]),
+                                     reinterpret_cast<float*>(ws + w.scale[3]), nullptr, nullptr, nullptr, 0, s);
+      if (rc != HBL_OK) break;
+    }
     rc = launch_gemm_tensor(reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]), T,
                             in_dims[xi], w_i8, out_dims[i], b->alpha7 + i, static_cast<__nv_bfloat16*>(ys[i]), nullptr, s);
     if (rc != HBL_OK) break;

@@ -200,7 +200,8 @@ def hbl_block_forward(inputs: dict, weights: dict, alpha7: torch.Tensor, hidden:
         workspace = new_workspace(hbl_block_workspace_bytes(T, hidden, ffn), dev)
     b = hbl_block_t()
     for n in ("attn_in", "o_in", "ffn_in", "down_in"):
-        setattr(b, "x_" + n, inputs[n].data_ptr())
+        t = inputs.get(n)                                    # no "down_in": the call chains SiLU(gate) * up into W_down
+        setattr(b, "x_" + n, t.data_ptr() if t is not None else None)
     for n in dims:
         setattr(b, "W" + n, weights[n].data_ptr())
         setattr(b, "y" + n, outputs[n].data_ptr())

@@ -95,3 +95,31 @@ def test_forward_glu_matches_oracle(T):
     rms = y2.pow(2).mean(1, keepdim=True).sqrt()
     assert torch.all((y.float() - y2).abs() <= 1e-2 * torch.maximum(y2.abs(), rms))
     assert (y.float() != y2).float().mean() <= 1e-2
+
+
+@pytest.mark.parametrize("T", [7, 300])
+def test_block_chains_the_feed_forward(T):
+    """hbl_block_forward without a down input: the down projection takes SiLU(ygate) * yup from the outputs the
+    same call has just written.  It must give what hbl_forward_glu gives on those two outputs, on either path,
+    and leave the other six outputs as the unchained call does."""
+    H, F = 512, 2048
+    seed = 41
+    ins = {"attn_in": wl.rows("gauss", seed, 10, H, 0, T, "bf16"), "o_in": wl.rows("attn_out", seed, 11, H, 0, T, "bf16"),
+           "ffn_in": wl.rows("gauss", seed, 12, H, 0, T, "bf16")}
+    shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "up": (F, H), "gate": (F, H), "down": (H, F)}
+    packed, alphas = {}, []
+    for i, (n, sh) in enumerate(shapes.items()):
+        p, a = hbl.hbl_quantize_weights(torch.from_numpy(wl.rows("latent", seed, 20 + i, sh[1], 0, sh[0], "f32")).cuda(), EPS)
+        packed[n] = p
+        alphas.append(a)
+    alpha7 = torch.cat(alphas)
+    dev = {k: to_dev(v, "bf16") for k, v in ins.items()}
+    for path in (hbl.PATH_AUTO, hbl.PATH_TENSOR):
+        outs = hbl.hbl_block_forward(dev, packed, alpha7, H, F, 4, EPS, path=path)
+        assert hbl.hbl_check_status() == 0
+        want_down = hbl.hbl_forward_glu(outs["gate"], outs["up"], packed["down"], alphas[6], H, 4, EPS, path=path)
+        assert torch.equal(outs["down"], want_down)
+        full = dict(dev, down_in=torch.zeros((T, F), dtype=torch.bfloat16, device="cuda"))
+        ref = hbl.hbl_block_forward(full, packed, alpha7, H, F, 4, EPS, path=path)
+        for n in ("q", "k", "v", "o", "up", "gate"):
+            assert torch.equal(outs[n], ref[n])
