@@ -260,7 +260,7 @@ def norm_quantize_point(K, T, torch, hbl, peaks, iters=None):
     ring = max(2, min(16, -(-RING_BYTES // per_call)))
     gen = torch.Generator(device="cuda").manual_seed(700 + K)
     xs = [torch.randn((T, K), device="cuda", generator=gen).bfloat16() for _ in range(ring)]
-    gain = torch.rand((K,), device="cuda", generator=gen) + 0.5
+    gain = (torch.rand((K,), device="cuda", generator=gen) + 0.5).bfloat16()     # bf16, as models store it
     codes = torch.empty((T, K), dtype=torch.int8, device="cuda")
     scale = torch.empty((T,), dtype=torch.float32, device="cuda")
     L = hbl.lib()
@@ -269,7 +269,7 @@ def norm_quantize_point(K, T, torch, hbl, peaks, iters=None):
     def call():
         x = xs[state["i"] % ring]
         state["i"] += 1
-        rc = L.hbl_norm_quantize_act(x.data_ptr(), gain.data_ptr(), 1e-5, T, K, 4, EPS, codes.data_ptr(), scale.data_ptr(),
+        rc = L.hbl_norm_quantize_act(x.data_ptr(), gain.data_ptr(), 1, 1e-5, T, K, 4, EPS, codes.data_ptr(), scale.data_ptr(),
                                      None, None, None)
         if rc != 0:
             raise RuntimeError(f"hbl_norm_quantize_act returned {rc}")

@@ -121,10 +121,11 @@ int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim,
  * LN is taken as  x' = x / sqrt(mean_k x^2 + norm_eps) * gain[k],  computed in fp32 and rounded once to
  * bf16 (the type activations are handed on in), and x' is what Eq. 3-7 then see.
  *   x         device, bf16 [tokens, in_dim];  in_dim 2048, 4096, 8192 or 16384 (HBL_ERR_SHAPE otherwise)
- *   gain      device, fp32 [in_dim], 16-byte aligned, caller-owned
+ *   gain      device, [in_dim], fp32 or bf16 as gain_dtype says (HBL_F32 / HBL_BF16), 16-byte aligned,
+ *             caller-owned; a bf16 gain halves what every token re-reads from L2 and is the faster of the two
  *   norm_eps  >= 0 (HBL_ERR_EPS otherwise); the transform is always on
  * Everything else as hbl_forward. */
-int hbl_forward_norm(const void* x, const float* gain, float norm_eps, int tokens, int in_dim,
+int hbl_forward_norm(const void* x, const void* gain, int gain_dtype, float norm_eps, int tokens, int in_dim,
                      const void* W_packed, const float* alpha, int out_dim, int bits, float eps, void* y,
                      void* workspace, size_t workspace_bytes, int path, void* stream);
 
@@ -214,9 +215,9 @@ int hbl_glu_quantize_act(const void* gate, const void* up, int tokens, int in_di
 
 /* The activation side of hbl_forward_norm alone: normalise, transform, quantize.  With xr_out != NULL
  * nothing is quantized and xr_out[T,K] fp32 receives H_m x' instead (the other outputs may then be NULL). */
-int hbl_norm_quantize_act(const void* x, const float* gain, float norm_eps, int tokens, int in_dim, int bits,
-                          float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out, float* xr_out,
-                          void* stream);
+int hbl_norm_quantize_act(const void* x, const void* gain, int gain_dtype, float norm_eps, int tokens, int in_dim,
+                          int bits, float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out,
+                          float* xr_out, void* stream);
 
 /* Eq. 3-6: transform (optional), per-token statistic, quantize.  codes_out: int8
  * [T,K], one code per byte; scale_out: fp32 [T] (s_t); codesum_out: int32 [T],

@@ -141,10 +141,10 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int group, in
 // What happens to the token before the transform sees it:
 //   PRE_NONE  nothing;
 //   PRE_NORM  RMS normalisation and a gain vector ("LN" of Eq. 7): x' = bf16(x * rsqrt(mean x^2 + norm_eps) * gain),
-//             aux = gain, fp32 [K];
+//             aux = gain [K], fp32 (PRE_NORM) or bf16 (PRE_NORM_BF16);
 //   PRE_GLU   the SwishGLU product that feeds W_down: x' = bf16(SiLU(x) * aux), aux = the other projection's
 //             output, bf16 [T, K] (x is the one that passes through SiLU).
-enum { PRE_NONE = 0, PRE_NORM = 1, PRE_GLU = 2 };
+enum { PRE_NONE = 0, PRE_NORM = 1, PRE_GLU = 2, PRE_NORM_BF16 = 3 };   // PRE_NORM_BF16: the same with a bf16 gain
 template <int M, int BITS, int PRE = PRE_NONE>
 __global__ void __launch_bounds__(Geometry<M>::THREADS, 768 / Geometry<M>::THREADS)
 fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
@@ -222,7 +222,7 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
         raw[c] = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
-    if constexpr (PRE == PRE_NORM) {
+    if constexpr (PRE == PRE_NORM || PRE == PRE_NORM_BF16) {
       // mean square of the token in fp32 (64 values per thread, then the group), one reciprocal
       // square root, then (x * rstd) * gain rounded once to bf16 -- the transform's exact +-1
       // products need bf16 inputs, and bf16 is the type a model hands activations on in.
@@ -243,12 +243,21 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
       const float ss = group_reduce<NT, false>(ss_lo + ss_hi, red_f, group, lane, warp_cta);
       const float rstd = __frcp_rn(__fsqrt_rn(__fmaf_rn(ss, 1.0f / (float)K, norm_eps)));
       const f32x2_t rstd2 = pack2(rstd, rstd);
-      const float* gp = static_cast<const float*>(aux) + (warp << 8) + (lane << 3);
+      const size_t goff = (size_t)(warp << 8) + (lane << 3);
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
-        const float4 g0 = __ldg(reinterpret_cast<const float4*>(gp + ((size_t)c << (M - 3))));
-        const float4 g1 = __ldg(reinterpret_cast<const float4*>(gp + ((size_t)c << (M - 3)) + 4));
-        const f32x2_t g2[4] = {pack2(g0.x, g0.y), pack2(g0.z, g0.w), pack2(g1.x, g1.y), pack2(g1.z, g1.w)};
+        f32x2_t g2[4];
+        if constexpr (PRE == PRE_NORM_BF16) {                 // half the bytes to fetch from L2 per token
+          const uint4 gb = __ldg(reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(aux) + goff + ((size_t)c << (M - 3))));
+          const uint32_t gw[4] = {gb.x, gb.y, gb.z, gb.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) g2[i] = pack2(__uint_as_float(gw[i] << 16), __uint_as_float(gw[i] & 0xFFFF0000u));
+        } else {
+          const float* gp = static_cast<const float*>(aux) + goff + ((size_t)c << (M - 3));
+          const float4 g0 = __ldg(reinterpret_cast<const float4*>(gp));
+          const float4 g1 = __ldg(reinterpret_cast<const float4*>(gp + 4));
+          g2[0] = pack2(g0.x, g0.y); g2[1] = pack2(g0.z, g0.w); g2[2] = pack2(g1.x, g1.y); g2[3] = pack2(g1.z, g1.w);
+        }
         uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -537,11 +546,14 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
 
 }  // namespace
 
-int launch_norm_act_quant_bf16(const void* x, const float* gain, float norm_eps, int T, int K, int bits, float eps,
-                               int8_t* codes, float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill,
-                               size_t zero_fill_words, cudaStream_t s) {
+int launch_norm_act_quant_bf16(const void* x, const void* gain, int gain_dtype, float norm_eps, int T, int K, int bits,
+                               float eps, int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
+                               int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s) {
 #define HBL_CASE(MM)                                                                                              \
   case (1 << MM):                                                                                                 \
+    if (gain_dtype == HBL_BF16)                                                                                   \
+      return bits == 8 ? launch_one<MM, 8, PRE_NORM_BF16>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps) \
+                       : launch_one<MM, 4, PRE_NORM_BF16>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps); \
     return bits == 8 ? launch_one<MM, 8, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps) \
                      : launch_one<MM, 4, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps);
   switch (K) {

@@ -226,8 +226,8 @@ int hbl_quantize_weights_rotated(const void* W_latent, int w_dtype, int out_dim,
 namespace {
 
 // Requirements of the fused normalisation: bf16 input, the transform on, a width the bf16 kernel has.
-int check_norm_args(int x_dtype, int in_dim, const float* gain, float norm_eps, int tokens) {
-  if (x_dtype != HBL_BF16) return HBL_ERR_FORMAT;
+int check_norm_args(int x_dtype, int in_dim, const void* gain, int gain_dtype, float norm_eps, int tokens) {
+  if (x_dtype != HBL_BF16 || (gain_dtype != HBL_F32 && gain_dtype != HBL_BF16)) return HBL_ERR_FORMAT;
   if (!is_pow2(in_dim)) return HBL_ERR_NOT_POW2;
   if (!act_quant_bf16_supported(in_dim)) return HBL_ERR_SHAPE;
   if (!(norm_eps >= 0.0f) || !isfinite(norm_eps)) return HBL_ERR_EPS;
@@ -238,7 +238,8 @@ int check_norm_args(int x_dtype, int in_dim, const float* gain, float norm_eps, 
 
 // hbl_forward, hbl_forward_norm (gain != nullptr: normalise first) and hbl_forward_glu (up != nullptr: x is
 // the gate projection, the layer's input is SiLU(x) * up).
-int forward_impl(const void* x, int x_dtype, const float* gain, float norm_eps, const void* up, int tokens, int in_dim,
+int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, float norm_eps, const void* up, int tokens,
+                 int in_dim,
                  const void* W_packed, const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y,
                  void* workspace, size_t workspace_bytes, int path, void* stream) {
   int rc = check_dims(tokens, in_dim, out_dim);
@@ -276,7 +277,7 @@ int forward_impl(const void* x, int x_dtype, const float* gain, float norm_eps, 
   int32_t* zf = stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr;
   const size_t zw = stream_path ? w.zero_words : 0;
   int32_t* cs = stream_path ? codesum : nullptr;             // only the streaming kernel needs the code sums
-  rc = gain ? launch_norm_act_quant_bf16(x, gain, norm_eps, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s)
+  rc = gain ? launch_norm_act_quant_bf16(x, gain, gain_dtype, norm_eps, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s)
        : up ? launch_glu_act_quant_bf16(x, up, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s)
             : launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale, cs, nullptr, zf, zw, s);
   if (rc != HBL_OK) {
@@ -298,16 +299,16 @@ extern "C" {
 int hbl_forward(const void* x, int x_dtype, int tokens, int in_dim, const void* W_packed,
                 const float* alpha, int out_dim, int bits, int use_hadamard, float eps, void* y,
                 void* workspace, size_t workspace_bytes, int path, void* stream) {
-  return forward_impl(x, x_dtype, nullptr, 0.f, nullptr, tokens, in_dim, W_packed, alpha, out_dim, bits, use_hadamard, eps,
+  return forward_impl(x, x_dtype, nullptr, HBL_F32, 0.f, nullptr, tokens, in_dim, W_packed, alpha, out_dim, bits, use_hadamard, eps,
                       y, workspace, workspace_bytes, path, stream);
 }
 
-int hbl_forward_norm(const void* x, const float* gain, float norm_eps, int tokens, int in_dim, const void* W_packed,
-                     const float* alpha, int out_dim, int bits, float eps, void* y, void* workspace,
+int hbl_forward_norm(const void* x, const void* gain, int gain_dtype, float norm_eps, int tokens, int in_dim,
+                     const void* W_packed, const float* alpha, int out_dim, int bits, float eps, void* y, void* workspace,
                      size_t workspace_bytes, int path, void* stream) {
-  const int rc = check_norm_args(HBL_BF16, in_dim, gain, norm_eps, tokens);
+  const int rc = check_norm_args(HBL_BF16, in_dim, gain, gain_dtype, norm_eps, tokens);
   if (rc != HBL_OK) return rc;
-  return forward_impl(x, HBL_BF16, gain, norm_eps, nullptr, tokens, in_dim, W_packed, alpha, out_dim, bits, 1, eps, y,
+  return forward_impl(x, HBL_BF16, gain, gain_dtype, norm_eps, nullptr, tokens, in_dim, W_packed, alpha, out_dim, bits, 1, eps, y,
                       workspace, workspace_bytes, path, stream);
 }
 
@@ -318,7 +319,7 @@ int hbl_forward_glu(const void* gate, const void* up, int tokens, int in_dim, co
   if (!act_quant_bf16_supported(in_dim)) return HBL_ERR_SHAPE;
   if (tokens > 0 && !up) return HBL_ERR_NULL;
   if (!aligned(up, 16)) return HBL_ERR_ALIGN;
-  return forward_impl(gate, HBL_BF16, nullptr, 0.f, up, tokens, in_dim, W_packed, alpha, out_dim, bits, 1, eps, y,
+  return forward_impl(gate, HBL_BF16, nullptr, HBL_F32, 0.f, up, tokens, in_dim, W_packed, alpha, out_dim, bits, 1, eps, y,
                       workspace, workspace_bytes, path, stream);
 }
 
@@ -342,13 +343,14 @@ int hbl_glu_quantize_act(const void* gate, const void* up, int tokens, int in_di
                                    nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
-int hbl_norm_quantize_act(const void* x, const float* gain, float norm_eps, int tokens, int in_dim, int bits, float eps,
-                          int8_t* codes_out, float* scale_out, int32_t* codesum_out, float* xr_out, void* stream) {
+int hbl_norm_quantize_act(const void* x, const void* gain, int gain_dtype, float norm_eps, int tokens, int in_dim,
+                          int bits, float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out, float* xr_out,
+                          void* stream) {
   int rc = check_dims(tokens, in_dim, 16);
   if (rc != HBL_OK) return rc;
   rc = check_quant_args(HBL_BF16, in_dim, bits, 1, eps);
   if (rc != HBL_OK) return rc;
-  rc = check_norm_args(HBL_BF16, in_dim, gain, norm_eps, tokens);
+  rc = check_norm_args(HBL_BF16, in_dim, gain, gain_dtype, norm_eps, tokens);
   if (rc != HBL_OK) return rc;
   if (tokens == 0) return HBL_OK;
   if (!x) return HBL_ERR_NULL;
@@ -359,7 +361,7 @@ int hbl_norm_quantize_act(const void* x, const float* gain, float norm_eps, int 
   } else if (!aligned(xr_out, 16)) {
     return HBL_ERR_ALIGN;
   }
-  return launch_norm_act_quant_bf16(x, gain, norm_eps, tokens, in_dim, bits, eps, codes_out, scale_out, codesum_out,
+  return launch_norm_act_quant_bf16(x, gain, gain_dtype, norm_eps, tokens, in_dim, bits, eps, codes_out, scale_out, codesum_out,
                                     xr_out, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 

@@ -67,10 +67,10 @@ bool act_quant_bf16_supported(int K);
 int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
                           int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
                           cudaStream_t s);
-// The same with the token RMS-normalised and multiplied by gain[K] (fp32, device) first ("LN" of Eq. 7).
-int launch_norm_act_quant_bf16(const void* x, const float* gain, float norm_eps, int T, int K, int bits, float eps,
-                               int8_t* codes, float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill,
-                               size_t zero_fill_words, cudaStream_t s);
+// The same with the token RMS-normalised and multiplied by gain[K] (fp32 or bf16, device) first ("LN" of Eq. 7).
+int launch_norm_act_quant_bf16(const void* x, const void* gain, int gain_dtype, float norm_eps, int T, int K, int bits,
+                               float eps, int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
+                               int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s);
 // The same with the token replaced by SiLU(gate) * up first (both bf16 [T, K]): the SwishGLU input of W_down.
 int launch_glu_act_quant_bf16(const void* gate, const void* up, int T, int K, int bits, float eps, int8_t* codes,
                               float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,

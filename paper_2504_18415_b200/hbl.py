@@ -74,8 +74,8 @@ def lib() -> C.CDLL:
         L.hbl_check_status.argtypes = [vp]
         L.hbl_hadamard_f32.argtypes = [vp, i, i, i, vp, vp]
         L.hbl_hadamard_bf16.argtypes = [vp, i, i, vp, vp]
-        L.hbl_forward_norm.argtypes = [vp, vp, f, i, i, vp, vp, i, i, f, vp, vp, sz, i, vp]
-        L.hbl_norm_quantize_act.argtypes = [vp, vp, f, i, i, i, f, vp, vp, vp, vp, vp]
+        L.hbl_forward_norm.argtypes = [vp, vp, i, f, i, i, vp, vp, i, i, f, vp, vp, sz, i, vp]
+        L.hbl_norm_quantize_act.argtypes = [vp, vp, i, f, i, i, i, f, vp, vp, vp, vp, vp]
         L.hbl_forward_glu.argtypes = [vp, vp, i, i, vp, vp, i, i, f, vp, vp, sz, i, vp]
         L.hbl_glu_quantize_act.argtypes = [vp, vp, i, i, i, f, vp, vp, vp, vp, vp]
         L.hbl_quantize_act.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp]
@@ -236,13 +236,13 @@ def hbl_hadamard_bf16(g: torch.Tensor, out: torch.Tensor | None = None) -> torch
 def hbl_forward_norm(x: torch.Tensor, gain: torch.Tensor, norm_eps: float, W_packed: torch.Tensor, alpha: torch.Tensor,
                      out_dim: int, bits: int, eps: float = 1e-5, y: torch.Tensor | None = None,
                      workspace: torch.Tensor | None = None, path: int = PATH_AUTO) -> torch.Tensor:
-    """hbl_forward with RMS normalisation and a gain vector fused in front of the transform (bf16 x, fp32 gain)."""
+    """hbl_forward with RMS normalisation and a gain vector fused in front of the transform (bf16 x; fp32 or bf16 gain)."""
     T, K = x.shape
     if y is None:
         y = torch.empty((T, out_dim), dtype=torch.bfloat16, device=x.device)
     if workspace is None:
         workspace = new_workspace(hbl_workspace_bytes(T, K, out_dim), x.device)
-    _check(lib().hbl_forward_norm(_ptr(x), _ptr(gain), norm_eps, T, K, _ptr(W_packed), _ptr(alpha), out_dim, bits, eps,
+    _check(lib().hbl_forward_norm(_ptr(x), _ptr(gain), _dt(gain), norm_eps, T, K, _ptr(W_packed), _ptr(alpha), out_dim, bits, eps,
                                   _ptr(y), _ptr(workspace), workspace.numel(), path, _stream()), "hbl_forward_norm")
     return y
 
@@ -283,13 +283,13 @@ def hbl_norm_quantize_act(x: torch.Tensor, gain: torch.Tensor, norm_eps: float, 
     T, K = x.shape
     if export_xr:
         xr = torch.empty((T, K), dtype=torch.float32, device=x.device)
-        _check(lib().hbl_norm_quantize_act(_ptr(x), _ptr(gain), norm_eps, T, K, bits, eps, None, None, None, _ptr(xr),
+        _check(lib().hbl_norm_quantize_act(_ptr(x), _ptr(gain), _dt(gain), norm_eps, T, K, bits, eps, None, None, None, _ptr(xr),
                                            _stream()), "hbl_norm_quantize_act")
         return xr
     codes = torch.empty((T, K), dtype=torch.int8, device=x.device)
     scale = torch.empty((T,), dtype=torch.float32, device=x.device)
     csum = torch.empty((T,), dtype=torch.int32, device=x.device)
-    _check(lib().hbl_norm_quantize_act(_ptr(x), _ptr(gain), norm_eps, T, K, bits, eps, _ptr(codes), _ptr(scale),
+    _check(lib().hbl_norm_quantize_act(_ptr(x), _ptr(gain), _dt(gain), norm_eps, T, K, bits, eps, _ptr(codes), _ptr(scale),
                                        _ptr(csum), None, _stream()), "hbl_norm_quantize_act")
     return codes, scale, csum
 

@@ -67,10 +67,11 @@ def test_argument_errors_come_before_any_launch(L):
     assert q(p, 0, 512, 512, -1.0, p, p, p, 1 << 20, n) == 7
     assert q(p, 0, 512, 512, 1e-5, p, p, p, 8, n) == 6
     assert L.hbl_hadamard_f32(p, 0, 4, 384, p, n) == 3
-    assert L.hbl_norm_quantize_act(p, p, -1.0, 4, 4096, 4, 1e-5, p, p, p, n, n) == 7      # norm_eps < 0
-    assert L.hbl_norm_quantize_act(p, n, 1e-5, 4, 4096, 4, 1e-5, p, p, p, n, n) == 1      # no gain
-    assert L.hbl_norm_quantize_act(p, p, 1e-5, 4, 1024, 4, 1e-5, p, p, p, n, n) == 2      # width without a fused kernel
-    assert L.hbl_forward_norm(p, p, 1e-5, 4, 384, p, p, 512, 4, 1e-5, p, p, 1 << 30, 0, n) == 3
+    assert L.hbl_norm_quantize_act(p, p, 0, -1.0, 4, 4096, 4, 1e-5, p, p, p, n, n) == 7   # norm_eps < 0
+    assert L.hbl_norm_quantize_act(p, n, 0, 1e-5, 4, 4096, 4, 1e-5, p, p, p, n, n) == 1   # no gain
+    assert L.hbl_norm_quantize_act(p, p, 5, 1e-5, 4, 4096, 4, 1e-5, p, p, p, n, n) == 10  # gain dtype
+    assert L.hbl_norm_quantize_act(p, p, 1, 1e-5, 4, 1024, 4, 1e-5, p, p, p, n, n) == 2   # width without a fused kernel
+    assert L.hbl_forward_norm(p, p, 0, 1e-5, 4, 384, p, p, 512, 4, 1e-5, p, p, 1 << 30, 0, n) == 3
     assert L.hbl_glu_quantize_act(p, n, 4, 4096, 4, 1e-5, p, p, p, n, n) == 1             # no `up`
     assert L.hbl_glu_quantize_act(p, p, 4, 1024, 4, 1e-5, p, p, p, n, n) == 2
     assert L.hbl_forward_glu(p, p, 4, 384, p, p, 512, 4, 1e-5, p, p, 1 << 30, 0, n) == 3

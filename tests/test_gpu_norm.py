@@ -25,14 +25,19 @@ def gain_vector(K, seed):
     return rng.uniform(0.25, 2.0, K).astype(np.float32)
 
 
+@pytest.mark.parametrize("gain_dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("K", [2048, 4096, 8192, 16384])
-def test_norm_transform_matches_oracle(K):
+def test_norm_transform_matches_oracle(K, gain_dtype):
     T = 37 if K <= 8192 else 9
     x = wl.rows("ffn_mid" if K >= 8192 else "attn_out", 500 + K, 1, K, 0, T, "bf16")
     g = gain_vector(K, K)
+    gd = torch.from_numpy(g).cuda()
+    if gain_dtype == "bf16":                                  # the oracle sees the gain the kernel sees
+        gd = gd.bfloat16()
+        g = gd.float().cpu().numpy()
     xn, _ = orc.rmsnorm_bf16(x, g, NORM_EPS)
     want = orc.hadamard(xn)
-    got = hbl.hbl_norm_quantize_act(to_dev(x, "bf16"), torch.from_numpy(g).cuda(), NORM_EPS, 4, EPS, export_xr=True)
+    got = hbl.hbl_norm_quantize_act(to_dev(x, "bf16"), gd, NORM_EPS, 4, EPS, export_xr=True)
     got = got.cpu().numpy().astype(np.float64)
     tol = 1e-4 * np.abs(want).max(axis=1, keepdims=True)
     assert np.all(np.abs(got - want) <= tol), float((np.abs(got - want) / tol).max())
@@ -89,6 +94,10 @@ def test_forward_norm_matches_oracle(T):
     y = hbl.hbl_forward_norm(to_dev(x, "bf16"), torch.from_numpy(g).cuda(), NORM_EPS, packed, alpha, N, 4, EPS)
     assert hbl.hbl_check_status() == 0
     xd, gd = to_dev(x, "bf16"), torch.from_numpy(g).cuda()
+    if T == 16:                                               # one of the cases with a bf16 gain
+        gd = gd.bfloat16()
+        g = gd.float().cpu().numpy()
+        y = hbl.hbl_forward_norm(xd, gd, NORM_EPS, packed, alpha, N, 4, EPS)
     xn, pre = orc.rmsnorm_bf16(x, g, NORM_EPS)
     xk, n_moved = reconcile_bf16_inputs(hbl.hbl_norm_quantize_act(xd, gd, NORM_EPS, 4, EPS, export_xr=True), xn, pre)
     assert n_moved <= 1e-3 * xn.size
