@@ -591,13 +591,8 @@ def main():
             if want(name, T_):
                 points.append(layer_point(name, kind, seed, K_, N_, bits, had, T_, torch=torch, hbl=hbl, peaks=peaks))
 
-        for T_ in (1, 16, 256, 4096):
-            L("config2_Wo_1p3B", "attn_out", 2, 2048, 2048, 4, True, T_)
-        for T_ in (1, 16, 1024):
-            L("config3_Wdown_1p3B", "ffn_mid", 3, 8192, 2048, 4, True, T_)
-        for N_ in (12288, 32768):
-            for T_ in ((16, 4096, 32768) if full else (16, 4096)):
-                L(f"config4_a8_N{N_}", "gauss", 4, 4096, N_, 8, False, T_)
+        # the activation-side kernels first: they are bound by instruction issue, and right after the
+        # millisecond-long contractions below the power cap still holds the clocks down
         if full:
             for K_ in (4096, 8192):
                 if want("transform_backward_bf16", 16384):
@@ -606,6 +601,13 @@ def main():
                     points.append(norm_quantize_point(K_, 16384, torch, hbl, peaks))
                 if want("glu_transform_quantize_int4", 16384):
                     points.append(glu_quantize_point(K_, 16384, torch, hbl, peaks))
+        for T_ in (1, 16, 256, 4096):
+            L("config2_Wo_1p3B", "attn_out", 2, 2048, 2048, 4, True, T_)
+        for T_ in (1, 16, 1024):
+            L("config3_Wdown_1p3B", "ffn_mid", 3, 8192, 2048, 4, True, T_)
+        for N_ in (12288, 32768):
+            for T_ in ((16, 4096, 32768) if full else (16, 4096)):
+                L(f"config4_a8_N{N_}", "gauss", 4, 4096, N_, 8, False, T_)
         for T_ in ((1, 4, 16, 64, 256, 1024, 4096, 16384, 65536) if full else (1, 16, 256, 4096)):
             if want("config5_block_7B", T_):
                 points.append(block_point(T_, torch, hbl, peaks))
