@@ -253,6 +253,41 @@ def backward_transform_point(K, T, torch, hbl, peaks, iters=None):
     return out
 
 
+def weight_quantize_point(N, K, dtype_name, torch, hbl, peaks, iters=None):
+    """Eq. 1-2 on one latent weight tensor: the absmean pass and the ternarise-and-pack pass each read the
+    tensor once (it is larger than what stays in L2 between them, or nearly), 1/4 byte per weight written.
+    L2-cold: a ring of distinct latent tensors larger than L2."""
+    dt = torch.float32 if dtype_name == "f32" else torch.bfloat16
+    esz = 4 if dtype_name == "f32" else 2
+    per_call = 2 * N * K * esz + N * K // 4
+    ring = max(2, min(8, -(-RING_BYTES // (N * K * esz))))
+    gen = torch.Generator(device="cuda").manual_seed(300 + N + K)
+    Ws = [(torch.randn((N, K), device="cuda", generator=gen) * 0.02).to(dt) for _ in range(ring)]
+    packed = torch.empty(hbl.hbl_packed_weight_bytes(N, K), dtype=torch.uint8, device="cuda")
+    alpha = torch.empty(1, dtype=torch.float32, device="cuda")
+    L = hbl.lib()
+    ws_bytes = int(L.hbl_quantize_weights_workspace_bytes(N, K))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    state = {"i": 0}
+
+    def call():
+        W = Ws[state["i"] % ring]
+        state["i"] += 1
+        rc = L.hbl_quantize_weights(W.data_ptr(), 0 if dtype_name == "f32" else 1, N, K, EPS, packed.data_ptr(),
+                                    alpha.data_ptr(), ws.data_ptr(), ws_bytes, None)
+        if rc != 0:
+            raise RuntimeError(f"hbl_quantize_weights -> {rc}")
+
+    ms = time_loop(call, iters or 30, 3, torch)
+    gbs = per_call / (ms * 1e-3) / 1e9
+    out = {"point": f"weight_quantize_{dtype_name}", "tokens": 0, "in": K, "out": N, "bits": 2, "hadamard": False,
+           "ms": round(ms, 5), "weights_per_s": round(N * K / (ms * 1e-3), 1), "tops": 0.0, "alg_gbs": round(gbs, 1),
+           "ring": ring, "graph": False, "bound": "hbm", "frac": round(gbs / peaks["hbm_gbs"], 4)}
+    del Ws
+    torch.cuda.empty_cache()
+    return out
+
+
 def norm_quantize_point(K, T, torch, hbl, peaks, iters=None):
     """RMS normalisation + transform + INT4 quantizer in one kernel (the activation side of hbl_forward_norm):
     2 B read + 1 B written per element, L2-cold (ring of inputs larger than L2)."""
@@ -594,6 +629,10 @@ def main():
         # the activation-side kernels first: they are bound by instruction issue, and right after the
         # millisecond-long contractions below the power cap still holds the clocks down
         if full:
+            for dtype_name in ("f32", "bf16"):
+                for N_, K_ in ((2048, 8192), (4096, 16384)):            # W_down of the 1.3B and the 7B configuration
+                    if want(f"weight_quantize_{dtype_name}", 0):
+                        points.append(weight_quantize_point(N_, K_, dtype_name, torch, hbl, peaks))
             for K_ in (4096, 8192):
                 if want("transform_backward_bf16", 16384):
                     points.append(backward_transform_point(K_, 16384, torch, hbl, peaks))

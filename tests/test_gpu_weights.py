@@ -63,6 +63,59 @@ def test_weight_quant_special_values():
     assert np.array_equal(hbl.hbl_unpack_weights(packed, N, K).cpu().numpy(), wt)
 
 
+def _signs(shape, seed):
+    return np.where(np.random.default_rng(seed).integers(0, 2, size=shape) == 1, 1.0, -1.0)
+
+
+@pytest.mark.parametrize("k", [1, 2, 77, 4095, 0x3FFFFF])
+def test_weight_quant_decisions_next_to_the_threshold_f32(k):
+    """Eq. 1-2 round W / (alpha + eps) half to even: the result changes exactly where the fp32 quotient passes
+    1/2.  The tensor is built so that alpha is known exactly (every group of four entries adds up to 4 a in
+    magnitude), d = alpha + eps = 1 + k 2^-23, and the first entry of each group sits on d / 2 or a few fp32
+    steps beside it; the oracle decides by the fp32 division."""
+    N, K = 16, 128
+    eps = 2.0 ** -17
+    d = 1.0 + k * 2.0 ** -23
+    a = d - eps
+    h = d / 2
+    mag = np.full(N * K, a)
+    steps = np.arange(N * K // 4) % 9 - 4                          # -4 .. 4 fp32 steps (2^-24) beside d / 2
+    x = h + steps * 2.0 ** -24
+    mag[0::4] = x
+    mag[1::4] = 0.75 - x
+    mag[2::4] = mag[3::4] = (4 * a - 0.75) / 2
+    assert np.array_equal(mag.astype(np.float32).astype(np.float64), mag)      # all exactly fp32
+    assert np.float32(np.float32(a) + np.float32(eps)) == np.float32(d)
+    W = (mag * _signs(mag.shape, k)).astype(np.float32).reshape(N, K)
+    packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), eps)
+    wt, al = orc.weight_quant(W, eps, 32)
+    assert al == np.float32(a) and alpha.item() == al
+    got = hbl.hbl_unpack_weights(packed, N, K).cpu().numpy()
+    assert np.array_equal(got, wt)
+    on_or_below = np.abs(W.reshape(-1)[0::4]) <= np.float32(h)                   # what the rounding rule implies
+    assert np.array_equal(wt.reshape(-1)[0::4] == 0, on_or_below)
+
+
+@pytest.mark.parametrize("eps", [2.0 ** -9, 2.0 ** -8, 3 * 2.0 ** -10, 1e-5, 2.0 ** -8 + 2.0 ** -20])
+def test_weight_quant_decisions_next_to_the_threshold_bf16(eps):
+    """The same for bf16 latents: alpha = 1/2 exactly, d / 2 = 1/4 + eps / 2 falls on or between bf16 values."""
+    N, K = 16, 384
+    mag = np.full(N * K, 0.5)
+    m = np.arange(N * K // 3) % 6 - 2                               # -2 .. 3 bf16 steps (2^-9) beside 1/4
+    mag[0::3] = 0.25 + m * 2.0 ** -9
+    mag[1::3] = 0.125 - m * 2.0 ** -9
+    mag[2::3] = 1.125
+    Wt = torch.from_numpy((mag * _signs(mag.shape, 5)).reshape(N, K)).to(torch.bfloat16)
+    W = Wt.float().numpy()
+    assert np.array_equal(np.abs(W.reshape(-1)).astype(np.float64), mag)         # all exactly bf16
+    packed, alpha = hbl.hbl_quantize_weights(Wt.cuda(), eps)
+    wt, al = orc.weight_quant(W, eps, 32)
+    assert al == 0.5 and alpha.item() == 0.5
+    assert np.array_equal(hbl.hbl_unpack_weights(packed, N, K).cpu().numpy(), wt)
+    half_d = np.float32(np.float32(0.5) + np.float32(eps)) / np.float32(2)
+    assert np.array_equal(wt.reshape(-1)[0::3] == 0, np.abs(W.reshape(-1)[0::3]) <= half_d)
+
+
 @pytest.mark.parametrize("N,K,dtype", [(144, 512, "f32"), (528, 2048, "f32"), (256, 8192, "bf16"), (2048, 4096, "f32")])
 def test_rotated_weight_quant(N, K, dtype):
     """Weight-and-activation rotation (the ablation's other variant): W H is ternarised instead of W.
