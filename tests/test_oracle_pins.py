@@ -210,6 +210,32 @@ def test_ternary_alpha_is_fp64_mean_rounded_once():
 
 
 # ------------------------------------------------------------------ contraction and rescale
+@pytest.mark.parametrize("k", [1, 2, 77, 4095, 0x3FFFFF])
+def test_ternary_decision_at_the_rounding_threshold(k):
+    """Eq. 1-2 with round-half-to-even: W_t = sign(w) exactly where |w| / (alpha + eps) rounds above 1/2, which
+    in exact arithmetic is |w| > (alpha + eps) / 2, a tie going to 0.  The tensor fixes alpha exactly (every
+    group of four magnitudes adds up to 4 a), makes alpha + eps = 1 + k 2^-23, and puts the first entry of each
+    group on the threshold or a few fp32 steps beside it.  Entries of magnitude ~1.6 d check the clip."""
+    N, K = 16, 128
+    eps = 2.0 ** -17
+    d = 1.0 + k * 2.0 ** -23
+    a, h = d - eps, d / 2
+    mag = np.full(N * K, a)
+    x = h + (np.arange(N * K // 4) % 9 - 4) * 2.0 ** -24
+    mag[0::4] = x
+    mag[1::4] = 0.75 - x
+    mag[2::4] = mag[3::4] = (4 * a - 0.75) / 2
+    assert np.array_equal(mag.astype(np.float32).astype(np.float64), mag)       # every entry is an fp32 value
+    sign = np.where(np.arange(N * K) % 3 == 0, -1.0, 1.0)
+    W = (mag * sign).astype(np.float32).reshape(N, K)
+    for prec in (32, 64):
+        wt, al = orc.weight_quant(W, eps, prec)
+        assert al == np.float32(a)
+        want = np.where(mag > h, sign, 0.0).astype(np.int8).reshape(N, K)
+        assert np.array_equal(wt, want)
+        assert np.count_nonzero(wt.reshape(-1)[0::4] == 0) > 100 and np.count_nonzero(wt.reshape(-1)[0::4]) > 100
+
+
 def test_gemm_matches_fp64_matmul_and_special_cases():
     rng = np.random.default_rng(11)
     q = rng.integers(-128, 128, size=(7, 96), dtype=np.int8)
