@@ -166,39 +166,35 @@ ternarise_pack_kernel(const void* __restrict__ W, int N, int K, float eps,
     if (n.kb >= n_kb) { n.kb -= n_kb; ++n.rg; }
     return n;
   };
-  auto fetch = [&](const Pos p, Turn& u) {       // p.g < n_groups
+  // No branch in fetch or emit: a group of padding rows (and a position past the end, fetched once before the
+  // loop stops) loads the tensor's last row instead and the result is replaced afterwards.
+  auto fetch = [&](const Pos p, Turn& u) {
     const int rb = (int)(p.rg / GPT), r0 = (int)(p.rg % GPT) * ROWS;
     const int R = rb * 128 + r0;
     u.inside = R < N;                                               // N % 16 == 0: a group is inside or outside
     u.dst = ((size_t)rb * n_kb + p.kb) * 1024 + (size_t)r0 * 4 + st_off;
-    if (u.inside) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const size_t row = (size_t)R + (BF16 ? 2 * j : j) + ld_row;
-        u.w[j] = __ldg(reinterpret_cast<const uint4*>(W) + ((row * K + (size_t)p.kb * 128) >> (BF16 ? 3 : 2)) + ld_vec);
-      }
+    for (int j = 0; j < 4; ++j) {
+      const int row = min(R + (BF16 ? 2 * j : j) + ld_row, N - 1);
+      u.w[j] = __ldg(reinterpret_cast<const uint4*>(W) + (((size_t)row * K + (size_t)p.kb * 128) >> (BF16 ? 3 : 2)) + ld_vec);
     }
   };
   auto emit = [&](const Turn& u) {
-    uint32_t k0 = 0x55555555u, k1 = 0x55555555u;                    // padding rows: w = 0
-    if (u.inside) {
-      uint32_t p[4];
+    uint32_t p[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if constexpr (BF16)
-          p[j] = (tern.four(make_uint2(u.w[j].x, u.w[j].y)) | (tern.four(make_uint2(u.w[j].z, u.w[j].w)) << 2)) << shift;
-        else
-          p[j] = tern.four(make_float4(__uint_as_float(u.w[j].x), __uint_as_float(u.w[j].y), __uint_as_float(u.w[j].z),
-                                       __uint_as_float(u.w[j].w))) << shift;
-      }
-      k0 = b0 ? p[2] : p[0];
-      k1 = b0 ? p[3] : p[1];
-      k0 |= __shfl_xor_sync(0xffffffffu, b0 ? p[0] : p[2], 1);
-      k1 |= __shfl_xor_sync(0xffffffffu, b0 ? p[1] : p[3], 1);
-      if constexpr (!BF16) k0 = (b1 ? k1 : k0) | __shfl_xor_sync(0xffffffffu, b1 ? k0 : k1, 2);
+    for (int j = 0; j < 4; ++j) {
+      if constexpr (BF16)
+        p[j] = (tern.four(make_uint2(u.w[j].x, u.w[j].y)) | (tern.four(make_uint2(u.w[j].z, u.w[j].w)) << 2)) << shift;
+      else
+        p[j] = tern.four(make_float4(__uint_as_float(u.w[j].x), __uint_as_float(u.w[j].y), __uint_as_float(u.w[j].z),
+                                     __uint_as_float(u.w[j].w))) << shift;
     }
-    packed[u.dst] = k0;
-    if constexpr (BF16) packed[u.dst + 8] = k1;                     // two rows further down
+    uint32_t k0 = b0 ? p[2] : p[0], k1 = b0 ? p[3] : p[1];
+    k0 |= __shfl_xor_sync(0xffffffffu, b0 ? p[0] : p[2], 1);
+    k1 |= __shfl_xor_sync(0xffffffffu, b0 ? p[1] : p[3], 1);
+    if constexpr (!BF16) k0 = (b1 ? k1 : k0) | __shfl_xor_sync(0xffffffffu, b1 ? k0 : k1, 2);
+    packed[u.dst] = u.inside ? k0 : 0x55555555u;                    // padding rows: w = 0
+    if constexpr (BF16) packed[u.dst + 8] = u.inside ? k1 : 0x55555555u;   // two rows further down
   };
   const size_t g_first = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
   Pos pos = {g_first, g_first / n_kb, (int)(g_first % n_kb)};
@@ -207,15 +203,13 @@ ternarise_pack_kernel(const void* __restrict__ W, int N, int K, float eps,
   fetch(pos, a);
   for (;;) {
     pos = advance(pos);
-    const bool more_b = pos.g < n_groups;
-    if (more_b) fetch(pos, b);
+    fetch(pos, b);
     emit(a);
-    if (!more_b) break;
+    if (pos.g >= n_groups) break;
     pos = advance(pos);
-    const bool more_a = pos.g < n_groups;
-    if (more_a) fetch(pos, a);
+    fetch(pos, a);
     emit(b);
-    if (!more_a) break;
+    if (pos.g >= n_groups) break;
   }
 }
 
