@@ -11,7 +11,7 @@
 //     lane eight consecutive bf16 values, which is exactly the A fragment of an
 //     m16n8k16 MMA; multiplied by the 16x16 matrix of +-1 (exact in bf16, fp32
 //     accumulation of exact products) two MMAs return the same eight positions
-//     transformed over index bits {0,1,3,4} -- including the two bits that live
+//     transformed over index bits {0,2,3,4} -- including the two bits that live
 //     in other lanes, so no shuffle is needed -- and already widened to fp32.
 //   * All other stages are packed fp32 butterflies (add/sub.f32x2: two
 //     butterflies per issue slot) on 64 elements held in registers.
@@ -175,7 +175,7 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   float* buf = smem + (size_t)group * K;
 
   // ---- the 16x16 sign matrix as B fragments (two MMAs: output columns 0-7 and 8-15) ----
-  // k-bit domain of the MMA: k0 = index bit 0, k1 k2 = index bits 3 4 (the lane's t), k3 = index bit 1.
+  // k-bit domain of the MMA: k0 = index bit 0, k1 k2 = index bits 3 4 (the lane's t), k3 = index bit 2.
   uint32_t hb[2][2];
   {
     const int t = lane & 3, g = lane >> 2;
@@ -272,20 +272,23 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
     }
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-      // A fragment: (x: m 0,1) rows g, k3 = 0; (z: m 4,5) rows g+8; (y: m 2,3) k3 = 1; (w: m 6,7) both
+      // A fragment, the loaded 16 bytes as they are: (x: m 0,1) rows g, k3 = 0; (y: m 2,3) rows g+8;
+      // (z: m 4,5) k3 = 1; (w: m 6,7) both.  No register has to move between the load and the MMA, and each
+      // MMA's four results are the two pairs that later leave in one 16-byte shared-memory store.
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         float d[4];
-        mma_bf16_16816(d, raw[c].x, raw[c].z, raw[c].y, raw[c].w, hb[j][0], hb[j][1]);
-        // d[2h + b] is position m = b + 2j + 4h; pair index p = j + 2h
-        v[c * 4 + j] = pack2(d[0], d[1]);
-        v[c * 4 + j + 2] = pack2(d[2], d[3]);
+        mma_bf16_16816(d, raw[c].x, raw[c].y, raw[c].z, raw[c].w, hb[j][0], hb[j][1]);
+        // d[2h + b] is position m = b + 2h + 4j; pair index p = h + 2j
+        v[c * 4 + 2 * j] = pack2(d[0], d[1]);
+        v[c * 4 + 2 * j + 1] = pack2(d[2], d[3]);
       }
     }
   }
-  // pair index e = c*4 + p: bit 0 = index bit 1 (done), bit 1 = index bit 2, bits 2..4 = the chunk bits
+  // pair index e = c*4 + p: bit 0 = index bit 1, bit 1 = index bit 2 (done by the MMA), bits 2..4 = the chunk bits
   const f32x2_t minus_one2 = opaque_minus_one2();
-  stages2<1, 5>(v, minus_one2);
+  stages2<0, 1>(v, minus_one2);
+  stages2<2, 5>(v, minus_one2);
 
   // ---- exchange ----
   // Swizzled addresses are (thread part) ^ (compile-time part); the two parts meet in bit 2
