@@ -79,7 +79,10 @@ size_t hbl_quantize_weights_workspace_bytes(int out_dim, int in_dim);
 /* Eq. 1-2.  W_latent: [out_dim, in_dim] row-major, fp32 or bf16.  Writes the
  * packed ternary tensor (hbl_packed_weight_bytes) and the fp32 alpha (device,
  * one float).  alpha is the fp64-accumulated mean rounded once to fp32; the
- * ternary decision is rint(W / (alpha + eps)) in IEEE fp32. */
+ * ternary decision is that of rint(W / (alpha + eps)) in IEEE fp32 with ties to
+ * even, clipped to [-1, 1] -- taken as |W| > (alpha + eps) / 2, which is the same
+ * decision for every fp32 (bf16) W.  A NaN weight becomes -1.  The tensor is read
+ * twice (absmean, then ternarise and pack); nothing else of its size is touched. */
 int hbl_quantize_weights(const void* W_latent, int w_dtype, int out_dim, int in_dim, float eps,
                          void* W_packed, float* alpha, void* workspace, size_t workspace_bytes,
                          void* stream);
