@@ -10,7 +10,7 @@ from parity_utils import EPS
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("N,K", [(16, 128), (512, 512), (2048, 2048), (528, 384), (2048, 8192)])
+@pytest.mark.parametrize("N,K", [(16, 128), (512, 512), (2048, 2048), (528, 384), (2048, 8192), (16, 32768), (1040, 1152)])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_weight_quant_is_bit_exact(N, K, dtype):
     W = wl.rows("latent", 11, N + K, K, 0, N, dtype)
