@@ -103,7 +103,7 @@ struct Ternary {
 // sign(w) exactly when fl(|w| / d) > 1/2, and that holds exactly when |w| > d / 2.  (d / 2 is exact in fp32;
 // |w| <= d/2 gives a quotient <= 1/2, which rounds to 0; the next fp32 value above d/2 is already more than
 // d/2 (1 + 2^-24), whose quotient lies above the midpoint between 1/2 and the next fp32 value, so it rounds
-// above 1/2 and then to 1.)  A NaN weight becomes -1, as the chain of fmax/fmin on the quotient made it.
+// above 1/2 and then to 1.)  A NaN weight becomes -1, which is what fmin(fmax(rint(NaN), -1), 1) gives.
 //
 // A warp takes a group of rows of one 128 x 128 tile at a time, 64 bytes per lane in four 16-byte loads.
 //   fp32: four rows; lane l loads columns 4l .. 4l+3 of each (one coalesced 512-byte request per row): byte
