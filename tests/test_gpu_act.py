@@ -115,6 +115,23 @@ def test_quantize_act_without_transform_is_bit_exact(bits):
         check_codes(codes.cpu().numpy(), q, v)
 
 
+@pytest.mark.parametrize("K,T", [(16384, 70), (32768, 65), (11008, 66), (384, 131), (128, 203), (2048, 1025)])
+@pytest.mark.parametrize("bits", [4, 8])
+def test_quantize_act_without_transform_wide_and_odd_widths(K, T, bits):
+    """bf16 rows of more than 64 tokens without the transform go through the row quantizer: the widest rows,
+    widths that are not powers of two, a width below one warp's share, ragged token counts."""
+    x = wl.rows("attn_out" if K < 8192 else "ffn_mid", 40 + bits, 1, K, 0, T, "bf16")
+    codes, scale, csum = hbl.hbl_quantize_act(to_dev(x, "bf16"), bits, False, EPS)
+    assert hbl.hbl_check_status() == 0
+    q, v, s, st = orc.act_quant(x.astype(np.float64), bits, EPS, 32)
+    cg = codes.cpu().numpy()
+    check_codes(cg, q, v)
+    assert np.allclose(scale.cpu().numpy(), s, rtol=2e-6, atol=0)
+    assert np.array_equal(csum.cpu().numpy(), cg.astype(np.int64).sum(1))
+    if bits == 8:
+        assert np.array_equal(cg, q)                      # the maximum is exact: identical decisions
+
+
 def test_quantize_act_generic_width_and_fp32_input():
     K, T = 384, 19                       # not a power of two: plain BitLinear input only
     x = wl.rows("gauss", 9, 1, K, 0, T, "f32")
