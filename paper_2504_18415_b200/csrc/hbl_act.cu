@@ -110,6 +110,16 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int group_war
 }
 
 constexpr float kSqrt7 = 2.6457513110645906f;
+constexpr float kMagicRound = 12582912.0f;          // 1.5 * 2^23: y + kMagicRound has rint(y) in its low mantissa bits
+
+// Four products -> four codes in one word: clamp, then round by the magic-number add (exact for |y| < 2^22, ties
+// to even; no float-to-int conversion, which issues at a quarter of the rate).  The same decisions as
+// clamp(rint(y)) for every finite y.
+__device__ __forceinline__ uint32_t codes4(float y0, float y1, float y2, float y3, float lo, float hi) {
+  const uint32_t a = __float_as_uint(fminf(fmaxf(y0, lo), hi) + kMagicRound), b = __float_as_uint(fminf(fmaxf(y1, lo), hi) + kMagicRound);
+  const uint32_t c = __float_as_uint(fminf(fmaxf(y2, lo), hi) + kMagicRound), d = __float_as_uint(fminf(fmaxf(y3, lo), hi) + kMagicRound);
+  return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
 
 // One CTA = TPC token groups of NT = K/E threads.
 template <int M, int E, bool HAD>
@@ -242,7 +252,7 @@ act_quant_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int bits, f
   }
   const float c = (bits == 8) ? 127.0f : kSqrt7;
   const float rq = __fdiv_rn(c, st + eps) * norm;
-  const int lo = (bits == 8) ? -128 : -8, hi = (bits == 8) ? 127 : 7;
+  const float lo = (bits == 8) ? -128.0f : -8.0f, hi = (bits == 8) ? 127.0f : 7.0f;
 
   // ---- quantize, pack 4 codes per word, store runs of RUN consecutive codes ----
   int csum = 0;
@@ -251,15 +261,9 @@ act_quant_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int bits, f
     uint32_t words[RUN / 4];
 #pragma unroll
     for (int w = 0; w < RUN / 4; ++w) {
-      uint32_t pk = 0;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        int q = __float2int_rn(v[j0 + w * 4 + i] * rq);
-        q = max(lo, min(hi, q));
-        csum += q;
-        pk |= (uint32_t)(q & 0xFF) << (8 * i);
-      }
-      words[w] = pk;
+      const int j = j0 + w * 4;
+      words[w] = codes4(v[j] * rq, v[j + 1] * rq, v[j + 2] * rq, v[j + 3] * rq, lo, hi);
+      csum = __dp4a((int)words[w], 0x01010101, csum);
     }
     if (live) {
       const int o = HAD ? LF::off(j0) : L0::off(j0);
@@ -333,18 +337,13 @@ act_quant_generic_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int
   if (bits != 8) st = st / (float)K;
   const float c = (bits == 8) ? 127.0f : kSqrt7;
   const float rq = __fdiv_rn(c, st + eps);
-  const int lo = (bits == 8) ? -128 : -8, hi = (bits == 8) ? 127 : 7;
+  const float lo = (bits == 8) ? -128.0f : -8.0f, hi = (bits == 8) ? 127.0f : 7.0f;
   int csum = 0;
   for (int k = tid * 4; k < K; k += 1024) {
     float f[4];
     load4(k, f);
-    uint32_t pk = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      int q = max(lo, min(hi, __float2int_rn(f[i] * rq)));
-      csum += q;
-      pk |= (uint32_t)(q & 0xFF) << (8 * i);
-    }
+    const uint32_t pk = codes4(f[0] * rq, f[1] * rq, f[2] * rq, f[3] * rq, lo, hi);
+    csum = __dp4a((int)pk, 0x01010101, csum);
     *reinterpret_cast<uint32_t*>(codes + token * K + k) = pk;
   }
   for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xffffffffu, csum, o);
@@ -365,8 +364,6 @@ act_quant_generic_kernel(const void* __restrict__ xin, int x_is_bf16, int T, int
 // every 8-byte store of codes is coalesced and the token is read once.  Rounding is the magic-number add
 // (x * rq + 1.5 * 2^23 has rint(x * rq) in its low mantissa bits: no float-to-int conversion, which runs at a
 // quarter of the rate); the INT8 maximum is taken on bf16 pairs (exact); the sum of codes is a byte dot product.
-constexpr float kMagicRound = 12582912.0f;          // 1.5 * 2^23
-
 __device__ __forceinline__ float fma_sat_f32(float a, float b, float c) {
   float r;
   asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
