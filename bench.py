@@ -288,6 +288,37 @@ def weight_quantize_point(N, K, dtype_name, torch, hbl, peaks, iters=None):
     return out
 
 
+def row_quantize_point(K, T, bits, torch, hbl, peaks, iters=None):
+    """Eq. 5-6 on bf16 activations without the transform (the inputs of the plain BitLinear projections and of the
+    INT8 configuration): 2 B read + 1 B written per element, L2-cold (ring of inputs larger than L2)."""
+    per_call = 3 * T * K
+    ring = max(2, min(16, -(-RING_BYTES // per_call)))
+    gen = torch.Generator(device="cuda").manual_seed(500 + K + bits)
+    xs = [torch.randn((T, K), device="cuda", generator=gen).bfloat16() for _ in range(ring)]
+    codes = [torch.empty((T, K), dtype=torch.int8, device="cuda") for _ in range(ring)]
+    scale = torch.empty((T,), dtype=torch.float32, device="cuda")
+    csum = torch.empty((T,), dtype=torch.int32, device="cuda")
+    L = hbl.lib()
+    state = {"i": 0}
+
+    def call():
+        r = state["i"] % ring
+        state["i"] += 1
+        rc = L.hbl_quantize_act(xs[r].data_ptr(), 1, T, K, bits, 0, EPS, codes[r].data_ptr(), scale.data_ptr(),
+                                csum.data_ptr(), None)
+        if rc != 0:
+            raise RuntimeError(f"hbl_quantize_act -> {rc}")
+
+    ms = time_loop(call, iters or 30, 3, torch)
+    gbs = per_call / (ms * 1e-3) / 1e9
+    out = {"point": f"row_quantize_int{bits}", "tokens": T, "in": K, "out": K, "bits": bits, "hadamard": False,
+           "ms": round(ms, 5), "tokens_per_s": round(T / (ms * 1e-3), 1), "tops": 0.0, "alg_gbs": round(gbs, 1),
+           "ring": ring, "graph": False, "bound": "hbm", "frac": round(gbs / peaks["hbm_gbs"], 4)}
+    del xs, codes
+    torch.cuda.empty_cache()
+    return out
+
+
 def norm_quantize_point(K, T, torch, hbl, peaks, iters=None):
     """RMS normalisation + transform + INT4 quantizer in one kernel (the activation side of hbl_forward_norm):
     2 B read + 1 B written per element, L2-cold (ring of inputs larger than L2)."""
@@ -633,6 +664,9 @@ def main():
                 for N_, K_ in ((2048, 8192), (4096, 16384)):            # W_down of the 1.3B and the 7B configuration
                     if want(f"weight_quantize_{dtype_name}", 0):
                         points.append(weight_quantize_point(N_, K_, dtype_name, torch, hbl, peaks))
+            for bits_ in (8, 4):
+                if want(f"row_quantize_int{bits_}", 32768):
+                    points.append(row_quantize_point(4096, 32768, bits_, torch, hbl, peaks))
             for K_ in (4096, 8192):
                 if want("transform_backward_bf16", 16384):
                     points.append(backward_transform_point(K_, 16384, torch, hbl, peaks))
