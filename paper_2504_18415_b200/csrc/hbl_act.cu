@@ -432,6 +432,12 @@ quant_rows_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, int K, int NT
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) st += __shfl_xor_sync(0xffffffffu, st, o);
   }
+  if constexpr (BITS != 8) {
+    // the widened values are not worth keeping across the reduction (64 registers): make the compiler
+    // widen again below
+#pragma unroll
+    for (int c = 0; c < 8; ++c) asm volatile("" : "+r"(raw[c].x), "+r"(raw[c].y), "+r"(raw[c].z), "+r"(raw[c].w));
+  }
   if (lane == 0) red_f[warp] = st;
   __syncthreads();
   st = red_f[warp0];
