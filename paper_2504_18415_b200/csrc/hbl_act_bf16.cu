@@ -238,6 +238,9 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
           ss2 = fma2(v2, v2, ss2);
         }
       }
+      // (the widened values are not kept across the reduction: the compiler is made to widen again below)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) asm volatile("" : "+r"(raw[c].x), "+r"(raw[c].y), "+r"(raw[c].z), "+r"(raw[c].w));
       float ss_lo, ss_hi;
       unpack2(ss2, ss_lo, ss_hi);
       const float ss = group_reduce<NT, false>(ss_lo + ss_hi, red_f, group, lane, warp_cta);
