@@ -185,12 +185,14 @@ int hbl_forward_host(const void* x_host /* host */, int x_dtype, int tokens, int
 /* Instrumentation (host-side state, not thread-safe).
  * hbl_launch_count: kernels this library has launched since it was loaded.
  * hbl_profile_events: start_events / stop_events are HOST arrays of n cudaEvent_t
- * handles owned by the caller; from now on the i-th launch of the selected kernel
+ * handles owned by the caller; from now on the i-th launch of kernel class `kernel`
  * (1 = activation transform+quantize of Eq. 3-6, 2 = contraction+rescale of Eq. 7,
  * 3 = weight unpack, 4 unused) is bracketed by cudaEventRecord(start[i]) /
  * cudaEventRecord(stop[i]) on the launch's stream, until n pairs are used.
- * kernel = 0 switches it off.  Returns the number of pairs the previous
- * selection used (>= 0), or -status on an argument error. */
+ * Each class has a slot of its own, so several can be bracketed during the same
+ * calls; n = 0 switches the class off, kernel = 0 all of them.  Returns the number
+ * of pairs the replaced slot (kernel = 0: all slots) had used, or -status on an
+ * argument error. */
 unsigned long long hbl_launch_count(void);
 int hbl_profile_events(void** start_events, void** stop_events, int n, int kernel);
 
@@ -254,7 +256,8 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
  *   - The call allocates and frees nothing.  The first call on each device looks up
  *     the array's device address (that device must be current); make that first
  *     call outside any stream capture.
- *   - Every call reuses the same array and clears the part it needs on `stream`
+ *   - Every call reuses the same array, which keeps the previous call's contents, and
+ *     clears the ready flags (the only part that must start at zero) on `stream`
  *     first.  Two calls that can overlap on the GPU (different streams, no ordering
  *     between them) race on it: order them. */
 int hbl_gemm_i32_static(const int8_t* codes, const int32_t* codesum, int tokens, int in_dim,

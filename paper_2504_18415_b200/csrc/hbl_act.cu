@@ -519,13 +519,7 @@ int launch_one(const void* x, int x_dtype, int T, int bits, float eps, int8_t* c
   constexpr int PAD = (NT < 32) ? NT : 0;
   const size_t smem = HAD ? sizeof(float) * TPC * (K + PAD) : 0;
   auto kern = act_quant_kernel<M, E, HAD>;
-  if (smem > 48 * 1024) {
-    static bool done = false;   // idempotent attribute; a race only repeats the call
-    if (!done) {
-      HBL_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      done = true;
-    }
-  }
+  if (smem > 48 * 1024) HBL_ALLOW_DYNAMIC_SMEM(kern, smem);
   const int grid = (T + TPC - 1) / TPC;
   profile_before(KERNEL_ACT, s);
   HBL_CUDA_OK(launch_dependent(kern, dim3(grid), dim3(THREADS), smem, s, x, (int)(x_dtype == HBL_BF16), T, bits, eps,

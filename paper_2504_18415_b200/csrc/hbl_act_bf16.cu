@@ -533,13 +533,7 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
   using G = Geometry<M>;
   const size_t smem = sizeof(float) * G::TPC * G::K;
   auto kern = fwht_quant_bf16_kernel<M, BITS, PRE>;
-  if (smem > 48 * 1024) {
-    static bool done = false;   // idempotent attribute; a race only repeats the call
-    if (!done) {
-      HBL_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-      done = true;
-    }
-  }
+  if (smem > 48 * 1024) HBL_ALLOW_DYNAMIC_SMEM(kern, smem);
   const int grid = (T + G::TPC - 1) / G::TPC;
   profile_before(KERNEL_ACT, s);
   HBL_CUDA_OK(launch_dependent(kern, dim3(grid), dim3(G::THREADS), smem, s, static_cast<const __nv_bfloat16*>(x), T, eps,

@@ -23,21 +23,36 @@ int* device_status_word() {
   return cached[dev];
 }
 
+int sm_count() {
+  static int cached[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 namespace {
 unsigned long long g_launches = 0;
-struct Profile { void** starts = nullptr; void** stops = nullptr; int n = 0, next = 0, kernel = 0; bool open = false; } g_prof;
+// One slot per kernel class, so that several classes can be bracketed during the same calls.
+struct Profile { void** starts = nullptr; void** stops = nullptr; int n = 0, next = 0; bool open = false; } g_prof[KERNEL_WEIGHT + 1];
 }
 void note_launch() { ++g_launches; }
 void profile_before(int kernel_id, cudaStream_t s) {
-  if (g_prof.kernel != kernel_id || g_prof.next >= g_prof.n) return;
-  cudaEventRecord(static_cast<cudaEvent_t>(g_prof.starts[g_prof.next]), s);
-  g_prof.open = true;
+  Profile& pr = g_prof[kernel_id];
+  if (pr.next >= pr.n) return;
+  cudaEventRecord(static_cast<cudaEvent_t>(pr.starts[pr.next]), s);
+  pr.open = true;
 }
 void profile_after(int kernel_id, cudaStream_t s) {
-  if (g_prof.kernel != kernel_id || !g_prof.open) return;
-  cudaEventRecord(static_cast<cudaEvent_t>(g_prof.stops[g_prof.next]), s);
-  g_prof.open = false;
-  ++g_prof.next;
+  Profile& pr = g_prof[kernel_id];
+  if (!pr.open) return;
+  cudaEventRecord(static_cast<cudaEvent_t>(pr.stops[pr.next]), s);
+  pr.open = false;
+  ++pr.next;
 }
 }  // namespace hbl
 
@@ -505,9 +520,15 @@ unsigned long long hbl_launch_count(void) { return g_launches; }
 int hbl_profile_events(void** start_events, void** stop_events, int n, int kernel) {
   if (n < 0 || kernel < 0 || kernel > KERNEL_WEIGHT) return -HBL_ERR_SHAPE;
   if (n > 0 && kernel != 0 && (!start_events || !stop_events)) return -HBL_ERR_NULL;
-  const int used = g_prof.next;
-  g_prof.starts = start_events; g_prof.stops = stop_events;
-  g_prof.n = (kernel == 0) ? 0 : n; g_prof.next = 0; g_prof.kernel = kernel; g_prof.open = false;
+  if (kernel == 0) {                                          // everything off
+    int used = 0;
+    for (Profile& pr : g_prof) { used += pr.next; pr = Profile(); }
+    return used;
+  }
+  Profile& pr = g_prof[kernel];
+  const int used = pr.next;
+  pr = Profile();
+  if (n > 0) { pr.starts = start_events; pr.stops = stop_events; pr.n = n; }
   return used;
 }
 

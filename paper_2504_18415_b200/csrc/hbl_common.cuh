@@ -27,10 +27,32 @@ inline bool is_pow2(long v) { return v > 0 && (v & (v - 1)) == 0; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// Per-device state: a process may drive several GPUs, and function attributes, SM counts and symbol
+// addresses belong to the device that is current when they are set or read.
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+  int dev = 0;
+  return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
+int sm_count();   // multiprocessors of the current device (148 if the query fails)
+
 #define HBL_CUDA_OK(expr)                         \
   do {                                            \
     cudaError_t _e = (expr);                      \
     if (_e != cudaSuccess) return HBL_ERR_CUDA;   \
+  } while (0)
+
+// Raises a kernel's dynamic shared-memory limit, once per device and per instantiation (the attribute is
+// idempotent, so a race between host threads only repeats the call).
+#define HBL_ALLOW_DYNAMIC_SMEM(kern, bytes)                                                                  \
+  do {                                                                                                       \
+    static bool _done[::hbl::kMaxDevices] = {};                                                              \
+    const int _dev = ::hbl::current_device();                                                                \
+    if (_dev < 0) return HBL_ERR_CUDA;                                                                       \
+    if (!_done[_dev]) {                                                                                      \
+      HBL_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes)));    \
+      _done[_dev] = true;                                                                                    \
+    }                                                                                                        \
   } while (0)
 
 // ---- programmatic dependent launch ----------------------------------------------

@@ -586,17 +586,6 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
-
 int pad_tokens(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 128)); }
 
 template <int T_PAD, int KBP>
@@ -604,11 +593,7 @@ int launch_variant(const CodeMaps& maps, const Params& p, int grid, cudaStream_t
   using GEO = Geo<T_PAD, KBP>;
   constexpr size_t smem = GEO::SMEM;
   auto kern = gemm_stream_kernel<T_PAD, KBP>;
-  static bool done = false;   // idempotent attribute; a race only repeats the call
-  if (!done) {
-    HBL_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    done = true;
-  }
+  HBL_ALLOW_DYNAMIC_SMEM(kern, smem);
   // Programmatic dependent launch: if the previous operation on the stream is a kernel that signals
   // griddepcontrol.launch_dependents (the activation kernels do), this kernel may start while it runs.
   profile_before(KERNEL_CONTRACT, s);

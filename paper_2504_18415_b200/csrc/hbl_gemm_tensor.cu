@@ -342,12 +342,7 @@ int launch_shape(const int8_t* codes, const float* scale, int T, int K, const in
   if (rc != HBL_OK) return rc;
   rc = make_map(&tmB, W_i8, N, K, BN);
   if (rc != HBL_OK) return rc;
-  static bool done = false;   // idempotent attribute; a race only repeats the call
-  if (!done) {
-    HBL_CUDA_OK(cudaFuncSetAttribute(gemm_tensor_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)Shape<BN>::SMEM_BYTES));
-    done = true;
-  }
+  HBL_ALLOW_DYNAMIC_SMEM(gemm_tensor_kernel<BN>, Shape<BN>::SMEM_BYTES);
   int* status = device_status_word();
   if (status == nullptr) return HBL_ERR_CUDA;
   const int n_tiles = ((T + BM - 1) / BM) * ((N + BN - 1) / BN);
@@ -365,12 +360,7 @@ int launch_shape(const int8_t* codes, const float* scale, int T, int K, const in
 int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
                        const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s) {
   if (T <= 0) return HBL_OK;
-  static int n_sm = 0;
-  if (n_sm == 0) {
-    int dev = 0;
-    HBL_CUDA_OK(cudaGetDevice(&dev));
-    HBL_CUDA_OK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-  }
+  const int n_sm = sm_count();
   // The narrow tile only pays on very small grids, where even twice as many tiles leave half of the SMs
   // idle (measured: 2048 x 2048 at 256 tokens 14.3 -> 12.8 us).  It costs about 1.5x per weight row (a
   // 128 x 128 x 32 MMA reads as much of the token block from shared memory as a 128 x 256 x 32 one), and at

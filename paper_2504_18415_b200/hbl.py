@@ -373,7 +373,7 @@ class KernelTimer:
         return self
 
     def __exit__(self, *exc):
-        self.used = lib().hbl_profile_events(None, None, 0, 0)
+        self.used = lib().hbl_profile_events(None, None, 0, self.kernel)
 
     def times_ms(self):
         torch.cuda.synchronize()

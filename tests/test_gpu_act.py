@@ -85,13 +85,17 @@ def test_hadamard_bf16_exact_cases_and_involution():
 @pytest.mark.parametrize("K", ALL_K)
 @pytest.mark.parametrize("bits", [4, 8])
 @pytest.mark.parametrize("had", [True, False])
-def test_quantize_act_matches_oracle(K, bits, had):
+@pytest.mark.parametrize("prec", [32, 64])
+def test_quantize_act_matches_oracle(K, bits, had, prec):
+    """prec = 32: the oracle takes the rounding decision in IEEE fp32, as the kernel does; prec = 64: in fp64
+    from the exact statistic, i.e. Eq. 5-6 as written.  The same rule holds against both: a code may differ
+    by one only where the pre-rounding value is within 1e-5 (relative to the boundary, absolute below 1) of it."""
     T = 67 if K <= 8192 else 11
     kind = "ffn_mid" if K >= 8192 else "attn_out"
     x = make_x(K, T, 7 * K + bits, kind)
     codes, scale, csum = hbl.hbl_quantize_act(to_dev(x, "bf16"), bits, had, EPS)
     xr = orc.hadamard(x) if had else x.astype(np.float64)
-    q, v, s, st = orc.act_quant(xr, bits, EPS, 32)
+    q, v, s, st = orc.act_quant(xr, bits, EPS, prec)
     cg = codes.cpu().numpy()
     check_codes(cg, q, v)
     assert np.allclose(scale.cpu().numpy(), s, rtol=2e-6, atol=0)

@@ -276,6 +276,37 @@ def test_rescale_rounds_once_to_bf16():
     assert np.array_equal(yb, want)
 
 
+def test_rescale_below_the_smallest_normal_bf16():
+    """Outputs below 2^-126 take the subnormal branch of the rounding: bf16 subnormals are the multiples of
+    2^-133 (7 fraction bits under an exponent of -126), ties go to the even multiple, and the top of the range
+    carries into the smallest normal.  Each expected value is written out from that definition; the last check
+    holds the whole branch against the fp32 -> bf16 conversion of a library on fp32-exact inputs."""
+    import torch
+    u = 2.0 ** -133                                        # spacing of bf16 subnormals
+    cases = [
+        (1, 1.0 * u, 0x0001), (1, 5.0 * u, 0x0005), (-1, 5.0 * u, 0x8005), (3, 9.0 * u, 27),
+        (1, 0.5 * u, 0x0000),                              # tie between 0 and u: even (0)
+        (1, 1.5 * u, 0x0002),                              # tie between u and 2u: even (2u)
+        (1, 2.5 * u, 0x0002),                              # tie between 2u and 3u: even (2u)
+        (1, 2.5 * u * (1 + 2.0 ** -30), 0x0003),           # just above that tie
+        (1, 0.49 * u, 0x0000), (-1, 0.49 * u, 0x8000),     # underflow keeps the sign
+        (1, 127.0 * u, 0x007F),                            # the largest subnormal
+        (1, 127.5 * u, 0x0080),                            # tie at the top: even = 128 u = 2^-126, the smallest normal
+        (1, 127.4 * u, 0x007F),
+        (1, 2.0 ** -126, 0x0080), (1, 2.0 ** -127, 0x0040),
+    ]
+    for a, s, bits in cases:
+        yb, y64 = orc.rescale(np.array([[a]], np.int32), np.array([s]), 1.0)
+        assert yb[0, 0] == bits, (a, s, hex(int(yb[0, 0])), hex(bits))
+        assert y64[0, 0] == a * s
+    rng = np.random.default_rng(11)
+    mant = rng.integers(1, 1 << 20, size=(1, 256)).astype(np.int32)            # fp32-exact subnormal products
+    yb, y64 = orc.rescale(mant, np.array([2.0 ** -146]), 1.0)                  # values in (0, 2^-126)
+    assert np.all(y64 < 2.0 ** -126) and np.array_equal(y64.astype(np.float32).astype(np.float64), y64)
+    want = torch.tensor(y64.astype(np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(yb, want)
+
+
 @pytest.mark.parametrize("prec", PRECS)
 @pytest.mark.parametrize("case", GOLD["layer"], ids=lambda c: c["cite"])
 def test_layer_hand_values(case, prec):

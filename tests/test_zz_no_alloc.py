@@ -17,6 +17,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import hbl_oracle as orc
 from paper_2504_18415_b200 import hbl, workloads as wl
 
 EPS = 1e-5
@@ -44,6 +45,9 @@ def test_static_scratch_matches_workspace_version_on_consecutive_calls():
         assert hbl.hbl_check_status() == 0
         assert torch.equal(got, want), f"call {n}: first static call differs"
         assert torch.equal(again, want), f"call {n}: second static call differs"
+        # and both are the exact integer contraction, as the CPU oracle computes it
+        wt = hbl.hbl_unpack_weights(packed, N, K).cpu().numpy()
+        assert np.array_equal(got.cpu().numpy(), orc.gemm(q.cpu().numpy(), wt)), f"call {n}: differs from the oracle"
 
 
 @pytest.mark.gpu
@@ -58,8 +62,8 @@ def test_sizes_beyond_the_fixed_array_are_refused_on_the_host():
     L = hbl.lib()
     p, n = C.c_void_p(1024), C.c_void_p(0)
     call = lambda T, K, N: L.hbl_gemm_i32_static(p, p, T, K, p, N, p, n)
-    assert call(65, 1024, 1024) == 11          # beyond the streaming kernel's token limit
-    assert call(64, 1024, 8192) == 11          # the fixed array holds slots for 16 tokens
+    assert call(65, 1024, 1024) == 11          # the fixed array holds slots for 16 tokens
+    assert call(64, 1024, 8192) == 11
     assert call(17, 1024, 1024) == 11
     assert call(16, 65536, 1024) == 11         # in_dim beyond the library's maximum
     assert call(16, 1000, 1024) == 2           # shape errors still come first
