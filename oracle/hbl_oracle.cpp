@@ -3,7 +3,9 @@
 // TEST INFRASTRUCTURE, not product: a plain, slow, step-by-step restatement of
 // the paper's definitions (Eq. 1-7: absmean ternary weights, the Sylvester
 // Hadamard recursion, per-token absmax-INT8 / absmean-INT4 activation
-// quantizers, the integer contraction and the rescale).  It shares no code with
+// quantizers, the integer contraction and the rescale; plus the normalisation and
+// gating product that feed the layer and the low-bit attention-state quantizer of
+// section 3.1, each marked where it is defined).  It shares no code with
 // the CUDA path and must only be used by the tests, the smoke check and the
 // benchmark's CPU-baseline leg.
 //
@@ -258,6 +260,53 @@ int orc_rescale(const int32_t* acc, const double* s, float alpha, long T, long N
             y_bits[t * N + o] = bf16_from_double(y);
         }
     return 0;
+}
+
+// Low-bit attention states (section 3.1, Tables 2-3): the Q, K and V heads are quantized after the rotary
+// embedding "to unsigned integers using the absmax function", and the K/V heads of the [BOS] token stay at
+// 8 bits.  The paper prints no formula; the reading taken is Eq. 5's absmax quantizer at b bits, one
+// statistic per head of each token, stored with an offset so that the code is unsigned:
+//     gamma = max_d |x[d]|,   q = RoundClip((2^(b-1) - 1) / (gamma + eps) * x, -2^(b-1), 2^(b-1) - 1),
+//     u = q + 2^(b-1)  in [0, 2^b - 1],   dequantization scale s = gamma / (2^(b-1) - 1).
+// (b = 8 is Eq. 5 itself plus the offset 128.)  Every choice here -- per-head granularity, the symmetric
+// grid, the offset -- is a reading: parity unpinned.
+// x: fp32 [R, D] (R = tokens * heads rows of one head each).  bits_row (may be null): bits per row, for the
+// rows kept at another width (the [BOS] token's heads at 8); otherwise `bits` for every row.
+// Outputs: u (uint8, one code per byte), v (fp64 pre-rounding values, may be null), s (fp64 [R]).
+int orc_kv_quant(const float* x, long R, long D, int bits, const int* bits_row, float eps, int prec,
+                 uint8_t* u, double* v_out, double* s_out) {
+    if (bits < 2 || bits > 8) return 4;
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (long r = 0; r < R; ++r) {
+        const int b = bits_row ? bits_row[r] : bits;
+        if (b < 2 || b > 8) { bad |= 1; continue; }
+        const double half = (double)(1 << (b - 1));            // 2^(b-1)
+        const double c = half - 1.0;
+        const float* row = x + r * D;
+        double gamma = 0.0;
+        for (long d = 0; d < D; ++d) gamma = std::fmax(gamma, std::fabs((double)row[d]));
+        if (prec == 32) {
+            const float g32 = (float)gamma;
+            const float rq = (float)c / (g32 + eps);
+            for (long d = 0; d < D; ++d) {
+                const float v = rq * row[d];
+                if (v_out) v_out[r * D + d] = (double)v;
+                const float q = std::fmin(std::fmax(round_half_even_f(v), (float)-half), (float)(half - 1.0));
+                u[r * D + d] = (uint8_t)((int)q + (int)half);
+            }
+            s_out[r] = (double)g32 / c;
+        } else {
+            const double rq = c / (gamma + (double)eps);
+            for (long d = 0; d < D; ++d) {
+                const double v = rq * (double)row[d];
+                if (v_out) v_out[r * D + d] = v;
+                u[r * D + d] = (uint8_t)((int)clipd(round_half_even(v), -half, half - 1.0) + (int)half);
+            }
+            s_out[r] = gamma / c;
+        }
+    }
+    return bad ? 4 : 0;
 }
 
 // The whole layer for T tokens against already-ternarised weights: Eq. 3-7 chained.

@@ -88,6 +88,21 @@ def swiglu_bf16(gate: np.ndarray, up: np.ndarray):
     return out, pre
 
 
+def kv_quant(x: np.ndarray, bits: int, eps: float = 1e-5, prec: int = 32, bits_row: np.ndarray | None = None):
+    """Section 3.1: absmax quantizer at `bits` bits, one statistic per row (= one head of one token), unsigned
+    codes u = q + 2^(bits-1).  x fp32 [R, D].  bits_row int32 [R] overrides the width per row (the [BOS] rows at 8).
+    Returns (u uint8 [R,D], v fp64 pre-rounding [R,D], s fp64 [R])."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    R, D = x.shape
+    u = np.empty((R, D), dtype=np.uint8)
+    v = np.empty((R, D), dtype=np.float64)
+    s = np.empty((R,), dtype=np.float64)
+    br = None if bits_row is None else np.ascontiguousarray(bits_row, dtype=np.int32)
+    _check(lib().orc_kv_quant(_p(x, C.c_float), C.c_long(R), C.c_long(D), C.c_int(bits), _p(br, C.c_int), C.c_float(eps),
+                              C.c_int(prec), _p(u, C.c_uint8), _p(v, C.c_double), _p(s, C.c_double)), "kv_quant")
+    return u, v, s
+
+
 def hadamard(x: np.ndarray) -> np.ndarray:
     """Eq. 3-4.  fp32 [T,K] -> fp64 [T,K], orthonormal, natural order."""
     x = np.ascontiguousarray(x, dtype=np.float32)

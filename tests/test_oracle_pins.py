@@ -505,3 +505,63 @@ def test_swiglu_derivative_and_single_rounding():
     assert np.array_equal(out, torch.from_numpy(out).bfloat16().float().numpy())
     ulp = 2.0 ** (np.floor(np.log2(np.abs(pre))) - 7)
     assert np.all(np.abs(out.astype(np.float64) - pre) <= ulp / 2 * (1 + 1e-12))
+
+
+# ------------------------------------------------------------------ low-bit attention states (section 3.1)
+@pytest.mark.parametrize("prec", PRECS)
+@pytest.mark.parametrize("case", GOLD["kv"], ids=lambda c: c["cite"][:40])
+def test_kv_hand_values(case, prec):
+    x = np.array([case["x"]], np.float32)
+    u, v, s = orc.kv_quant(x, case["bits"], case.get("eps", EPS), prec)
+    assert u[0].tolist() == case["u"]
+    assert abs(s[0] - case["s"]) <= 1e-6 * max(1.0, case["s"])
+
+
+@pytest.mark.parametrize("prec", PRECS)
+def test_kv_at_8_bits_is_eq5_plus_the_offset(prec):
+    """b = 8 must reduce to the (separately pinned) absmax INT8 quantizer of Eq. 5, head by head."""
+    x = wl.rows("gauss", 91, 1, 128, 0, 96, "bf16")
+    u, v, s = orc.kv_quant(x, 8, EPS, prec)
+    q, v8, s8, st = orc.act_quant(x.astype(np.float64), 8, EPS, prec)
+    assert np.array_equal(u.astype(np.int32) - 128, q.astype(np.int32))
+    assert np.array_equal(s, s8) and np.array_equal(v, v8)
+
+
+@pytest.mark.parametrize("bits", [3, 4, 8])
+def test_kv_invariants(bits):
+    """What the grid fixes whatever the data: the code range, the unreachable lowest code, the extreme element
+    landing on the outermost level, the dequantization error bound of a symmetric grid, sign symmetry, scale
+    equivariance and row independence (one statistic per head, not per token)."""
+    half = 1 << (bits - 1)
+    x = wl.rows("attn_out", 92, 1, 128, 0, 64, "bf16")
+    u, v, s = orc.kv_quant(x, bits, EPS, 64)
+    assert u.min() >= 1 and u.max() <= 2 * half - 1               # q = -2^(b-1) is never reached: |v| < 2^(b-1) - 1
+    amax = np.abs(x).argmax(axis=1)
+    rows = np.arange(x.shape[0])
+    want_top = np.where(x[rows, amax] > 0, 2 * half - 1, 1)
+    assert np.array_equal(u[rows, amax], want_top)
+    deq = (u.astype(np.float64) - half) * s[:, None]
+    gamma = np.abs(x).max(axis=1)
+    assert np.all(np.abs(deq - x) <= 0.5 * s[:, None] + gamma[:, None] * 2e-5)   # half a step (+ the eps shrink)
+    um, _, sm = orc.kv_quant(-x, bits, EPS, 64)
+    assert np.array_equal(um.astype(np.int32) - half, -(u.astype(np.int32) - half)) and np.array_equal(sm, s)
+    # a power-of-two rescale of one head changes that head's scale only (eps is negligible at this magnitude)
+    y = x.copy(); y[3] *= 4.0
+    u4, _, s4 = orc.kv_quant(y, bits, 1e-12, 64)
+    u1, _, s1 = orc.kv_quant(x, bits, 1e-12, 64)
+    assert np.array_equal(u4, u1) and s4[3] == 4.0 * s1[3] and np.array_equal(np.delete(s4, 3), np.delete(s1, 3))
+
+
+def test_kv_mixed_widths_and_bad_arguments():
+    """The [BOS] rows keep 8 bits: a per-row width must give each row exactly what a uniform call gives it."""
+    x = wl.rows("gauss", 93, 1, 64, 0, 12, "bf16")
+    br = np.array([8, 8, 3, 3, 3, 3, 8, 8, 3, 3, 3, 3], np.int32)
+    u, v, s = orc.kv_quant(x, 3, EPS, 32, bits_row=br)
+    u3, _, s3 = orc.kv_quant(x, 3, EPS, 32)
+    u8, _, s8 = orc.kv_quant(x, 8, EPS, 32)
+    assert np.array_equal(u[br == 3], u3[br == 3]) and np.array_equal(u[br == 8], u8[br == 8])
+    assert np.array_equal(s[br == 3], s3[br == 3]) and np.array_equal(s[br == 8], s8[br == 8])
+    with pytest.raises(RuntimeError):
+        orc.kv_quant(x, 9, EPS, 32)
+    with pytest.raises(RuntimeError):
+        orc.kv_quant(x, 1, EPS, 32)
