@@ -364,6 +364,36 @@ def row_quantize_point(K, T, bits, torch, hbl, peaks, iters=None):
     return out
 
 
+def kv_quantize_point(T, H, D, bits, torch, hbl, peaks, iters=None):
+    """The low-bit attention-state quantizer (absmax per head, unsigned codes): 2 B read + bits/8 B written per
+    element, L2-cold (ring of inputs larger than L2)."""
+    per_call = T * H * D * 2 + T * H * D * bits // 8 + 4 * T * H
+    ring = max(2, min(16, -(-RING_BYTES // per_call)))
+    gen = torch.Generator(device="cuda").manual_seed(1000 + bits)
+    xs = [torch.randn((T, H, D), device="cuda", generator=gen).bfloat16() for _ in range(ring)]
+    codes = torch.empty((T * H, D * bits // 8), dtype=torch.uint8, device="cuda")
+    scale = torch.empty((T * H,), dtype=torch.float32, device="cuda")
+    L = hbl.lib()
+    state = {"i": 0}
+
+    def call():
+        x = xs[state["i"] % ring]
+        state["i"] += 1
+        rc = L.hbl_quantize_kv(x.data_ptr(), T, H, D, bits, 0, EPS, codes.data_ptr(), scale.data_ptr(), None, None, None)
+        if rc != 0:
+            raise RuntimeError(f"hbl_quantize_kv -> {rc}")
+
+    ms = time_loop(call, iters or 30, 3, torch)
+    gbs = per_call / (ms * 1e-3) / 1e9
+    out = {"point": f"kv_quantize_int{bits}", "tokens": T, "in": H * D, "out": H * D, "bits": bits, "hadamard": False,
+           "ms": round(ms, 5), "tokens_per_s": round(T / (ms * 1e-3), 1), "tops": 0.0, "alg_gbs": round(gbs, 1),
+           "ring": ring, "graph": False, "bound": "hbm", "frac": round(gbs / peaks["hbm_gbs"], 4),
+           "frac_of_nominal_hbm": round(gbs / NOMINAL_HBM_GBS, 4)}
+    del xs
+    torch.cuda.empty_cache()
+    return out
+
+
 def norm_quantize_point(K, T, torch, hbl, peaks, iters=None):
     """RMS normalisation + transform + INT4 quantizer in one kernel (the activation side of hbl_forward_norm):
     2 B read + 1 B written per element, L2-cold (ring of inputs larger than L2)."""
@@ -719,6 +749,9 @@ def main():
             for bits_ in (8, 4):
                 if want(f"row_quantize_int{bits_}", 32768):
                     points.append(row_quantize_point(4096, 32768, bits_, torch, hbl, peaks))
+            for bits_ in (3, 4):
+                if want(f"kv_quantize_int{bits_}", 16384):
+                    points.append(kv_quantize_point(16384, 32, 128, bits_, torch, hbl, peaks))    # one of K / V of the 7B shape
             for K_ in (4096, 8192):
                 if want("transform_backward_bf16", 16384):
                     points.append(backward_transform_point(K_, 16384, torch, hbl, peaks))

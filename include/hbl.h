@@ -40,7 +40,7 @@ typedef enum {
   HBL_ERR_NULL = 1,        /* a required pointer is NULL */
   HBL_ERR_SHAPE = 2,       /* a dimension is negative, zero where not allowed, or not a supported multiple */
   HBL_ERR_NOT_POW2 = 3,    /* use_hadamard with in_dim not a power of two (Eq. 4 needs n = 2^m) */
-  HBL_ERR_BITS = 4,        /* bits not 4 or 8 */
+  HBL_ERR_BITS = 4,        /* bits not 4 or 8 (hbl_quantize_kv: not 3, 4 or 8) */
   HBL_ERR_ALIGN = 5,       /* a pointer is not aligned as required */
   HBL_ERR_WORKSPACE = 6,   /* workspace smaller than hbl_workspace_bytes() says */
   HBL_ERR_EPS = 7,         /* eps <= 0 or not finite */
@@ -262,6 +262,29 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
  *     between them) race on it: order them. */
 int hbl_gemm_i32_static(const int8_t* codes, const int32_t* codesum, int tokens, int in_dim,
                         const void* W_packed, int out_dim, int32_t* acc_out, void* stream);
+
+/* Low-bit attention states (section 3.1 "Inference", Tables 2-3): the Q, K and V heads are quantized after the
+ * rotary embedding "to unsigned integers using the absmax function" (4-bit, or 3-bit for the KV cache), and the
+ * K/V heads of the [BOS] token are kept at 8 bits.  The paper prints no formula; the one used is Eq. 5's absmax
+ * quantizer at b bits with one statistic per head of each token, stored with an offset so that it is unsigned:
+ *   gamma = max_d |x[d]|,  q = RoundClip((2^(b-1) - 1) / (gamma + eps) * x, -2^(b-1), 2^(b-1) - 1),
+ *   u = q + 2^(b-1) in [1, 2^b - 1],  scale = gamma / (2^(b-1) - 1),  so that  x ~ scale * (u - 2^(b-1)).
+ * The decision is taken in IEEE fp32 in the order written (division, product, round-half-to-even, clip).
+ *   x          device, bf16 [tokens, n_heads, head_dim] contiguous (the states after RoPE), 16-byte aligned
+ *   head_dim   64, 128 or 256 (HBL_ERR_SHAPE otherwise);  bits 3, 4 or 8 (HBL_ERR_BITS otherwise);  eps > 0
+ *   codes      device, written: hbl_kv_codes_bytes() bytes, 16-byte aligned.  Each head is a run of
+ *              head_dim * bits / 8 bytes; element d of the head is the bits [bits * d, bits * d + bits) of that
+ *              run read as a little-endian bit string (4 bits: element 2j in the low nibble of byte j)
+ *   scale      device, written: fp32 [tokens * n_heads]
+ *   bos_codes  device or NULL.  Not NULL: tokens t with t % seq_len == 0 (seq_len > 0: the first token of each
+ *              sequence of a [n_seq, seq_len] batch) are the [BOS] tokens; their heads are quantized at 8 bits
+ *              as well, into bos_codes [ceil(tokens / seq_len), n_heads, head_dim] (one byte per element) and
+ *              bos_scale [ceil(tokens / seq_len) * n_heads]; a reader of the cache takes these for position 0
+ * All buffers are the caller's; asynchronous on `stream`; nothing is allocated.  hbl_kv_codes_bytes returns 0
+ * for an unsupported shape. */
+size_t hbl_kv_codes_bytes(int tokens, int n_heads, int head_dim, int bits);
+int hbl_quantize_kv(const void* x, int tokens, int n_heads, int head_dim, int bits, int seq_len, float eps, void* codes,
+                    float* scale, void* bos_codes, float* bos_scale, void* stream);
 
 /* Packed ternary -> int8 [N,K] row-major, values in {-1,0,1}. */
 int hbl_unpack_weights(const void* W_packed, int out_dim, int in_dim, int8_t* w_out, void* stream);

@@ -165,7 +165,7 @@ const char* hbl_status_string(int status) {
     case HBL_ERR_NULL: return "null pointer";
     case HBL_ERR_SHAPE: return "unsupported shape";
     case HBL_ERR_NOT_POW2: return "in_dim must be a power of two for the Hadamard transform";
-    case HBL_ERR_BITS: return "bits must be 4 or 8";
+    case HBL_ERR_BITS: return "unsupported bit width";
     case HBL_ERR_ALIGN: return "misaligned pointer";
     case HBL_ERR_WORKSPACE: return "workspace too small";
     case HBL_ERR_EPS: return "eps must be positive and finite";
@@ -682,6 +682,28 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
   return run_gemm(p, codes, nullptr, codesum, tokens, in_dim, W_packed, out_dim, nullptr, nullptr, acc_out,
                   reinterpret_cast<int32_t*>(ws + w.acc), reinterpret_cast<int*>(ws + w.counters),
                   reinterpret_cast<int8_t*>(ws + w.w_i8), s);
+}
+
+size_t hbl_kv_codes_bytes(int tokens, int n_heads, int head_dim, int bits) {
+  if (tokens < 0 || n_heads <= 0 || (head_dim != 64 && head_dim != 128 && head_dim != 256)) return 0;
+  if (bits != 3 && bits != 4 && bits != 8) return 0;
+  return (size_t)tokens * n_heads * head_dim * bits / 8;
+}
+
+int hbl_quantize_kv(const void* x, int tokens, int n_heads, int head_dim, int bits, int seq_len, float eps, void* codes,
+                    float* scale, void* bos_codes, float* bos_scale, void* stream) {
+  if (tokens < 0 || n_heads <= 0) return HBL_ERR_SHAPE;
+  if (head_dim != 64 && head_dim != 128 && head_dim != 256) return HBL_ERR_SHAPE;
+  if (bits != 3 && bits != 4 && bits != 8) return HBL_ERR_BITS;
+  if (!(eps > 0.0f) || !isfinite(eps)) return HBL_ERR_EPS;
+  if (seq_len < 0 || (bos_codes != nullptr && seq_len == 0)) return HBL_ERR_SHAPE;
+  if (tokens == 0) return HBL_OK;
+  if (!x || !codes || !scale) return HBL_ERR_NULL;
+  if (bos_codes != nullptr && !bos_scale) return HBL_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(codes, 16) || !aligned(scale, 4) || !aligned(bos_codes, 16) || !aligned(bos_scale, 4))
+    return HBL_ERR_ALIGN;
+  return launch_kv_quant(x, (long)tokens * n_heads, n_heads, head_dim, bits, seq_len, eps, codes, scale, bos_codes, bos_scale,
+                         static_cast<cudaStream_t>(stream));
 }
 
 int hbl_unpack_weights(const void* W_packed, int out_dim, int in_dim, int8_t* w_out, void* stream) {

@@ -103,6 +103,9 @@ int launch_hadamard_bf16(const void* x, int T, int K, void* out, cudaStream_t s)
 int launch_weight_quant(const void* W, int w_dtype, int N, int K, float eps, void* packed, float* alpha,
                         void* ws, cudaStream_t s);
 int launch_unpack_weights(const void* packed, int N, int K, int8_t* out, cudaStream_t s);
+// Low-bit attention states (section 3.1): absmax quantizer at 3, 4 or 8 bits per head of each token, unsigned codes.
+int launch_kv_quant(const void* x, long n_rows, int n_heads, int head_dim, int bits, int seq_len, float eps, void* codes,
+                    float* scale, void* bos_codes, float* bos_scale, cudaStream_t s);
 // Contraction + epilogue.  Exactly one of y / acc_out is written.
 struct GemmSegment {          // one weight tensor of a (possibly fused) projection
   const void* W;              // packed (stream path) or int8 row-major (tensor path)

@@ -1,0 +1,153 @@
+// Low-bit attention states (BitNet v2, section 3.1, Tables 2-3): the Q, K and V heads are quantized after the
+// rotary embedding to unsigned integers with the absmax function, 4-bit or 3-bit for the KV cache, and the K/V
+// heads of the [BOS] token stay at 8 bits.  The paper prints no formula for it; this is Eq. 5's absmax quantizer
+// at b bits, one statistic per head of each token, stored with an offset so that the code is unsigned:
+//
+//   gamma = max_d |x[d]|,  q = RoundClip((2^(b-1) - 1) / (gamma + eps) * x, -2^(b-1), 2^(b-1) - 1),
+//   u = q + 2^(b-1),       s = gamma / (2^(b-1) - 1)          (x ~ s * (u - 2^(b-1)))
+//
+// Bound by HBM: 2 bytes read and b/8 bytes written per element.  A thread takes 8 consecutive elements of one
+// head (one 16-byte load), the head_dim / 8 lanes of a head share the maximum by shuffles, and the codes of a
+// head leave as one contiguous run of head_dim * b / 8 bytes.
+#include "hbl_common.cuh"
+
+namespace hbl {
+namespace {
+
+constexpr int kThreads = 256;
+
+constexpr int kUnroll = 4;                                   // 16-byte chunks in flight per thread
+constexpr float kMagic = 12582912.0f;                        // 1.5 * 2^23: x + kMagic has rint(x) in its low mantissa bits
+
+// Codes of 8 consecutive elements for width BITS, from the fp32 values f and the head's maximum g.
+// IEEE fp32, operations in the order the formula is written: c / (g + eps), times x, round to nearest even, clip.
+// (Clipping to the integer bounds first and rounding by the magic-number add gives the same integers as
+// rounding first: the bounds are integers and |v| is far below 2^22.)
+template <int BITS>
+__device__ __forceinline__ void codes8(const float (&f)[8], float g, float eps, uint32_t (&u)[8]) {
+  constexpr int HALF = 1 << (BITS - 1);
+  const float rq = __fdiv_rn((float)(HALF - 1), __fadd_rn(g, eps));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float v = fminf(fmaxf(__fmul_rn(rq, f[i]), (float)-HALF), (float)(HALF - 1));
+    u[i] = (__float_as_uint(__fadd_rn(v, kMagic + (float)HALF))) & 0xFFu;      // rint(v) + HALF, in [0, 2 HALF - 1]
+  }
+}
+
+// LPH = lanes per head = head_dim / 8.  A thread block takes tiles of kUnroll x kThreads chunks; a thread's
+// kUnroll loads are issued before any arithmetic.
+template <int BITS, int LPH>
+__global__ void __launch_bounds__(kThreads)
+kv_quant_kernel(const uint4* __restrict__ x, long n_rows, int n_heads, int seq_len, float eps,
+                unsigned char* __restrict__ codes, float* __restrict__ scale, unsigned char* __restrict__ bos_codes,
+                float* __restrict__ bos_scale) {
+  constexpr int HALF = 1 << (BITS - 1);
+  constexpr int ROW_BYTES = LPH * BITS;                     // head_dim * BITS / 8
+  constexpr long TILE = (long)kUnroll * kThreads;
+  const long n_chunks = n_rows * LPH;                       // (a multiple of LPH: a head is live or dead as a whole)
+  const int lane_in_head = threadIdx.x % LPH;
+  for (long tile0 = (long)blockIdx.x * TILE; tile0 < n_chunks; tile0 += (long)gridDim.x * TILE) {
+    uint4 raw[kUnroll];
+#pragma unroll
+    for (int k = 0; k < kUnroll; ++k) {
+      const long chunk = tile0 + k * kThreads + threadIdx.x;
+      raw[k] = chunk < n_chunks ? __ldg(x + chunk) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int k = 0; k < kUnroll; ++k) {
+      const long chunk = tile0 + k * kThreads + threadIdx.x;
+      const bool live = chunk < n_chunks;
+      const long row = (live ? chunk : n_chunks - 1) / LPH;
+      const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+      float f[8];
+      float m = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        m = fmaxf(m, fmaxf(fabsf(f[2 * i]), fabsf(f[2 * i + 1])));
+      }
+#pragma unroll
+      for (int o = LPH / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+
+      uint32_t u[8];
+      codes8<BITS>(f, m, eps, u);
+      unsigned char* dst = codes + row * ROW_BYTES;
+      if constexpr (BITS == 8) {
+        const uint2 o = make_uint2(u[0] | (u[1] << 8) | (u[2] << 16) | (u[3] << 24), u[4] | (u[5] << 8) | (u[6] << 16) | (u[7] << 24));
+        if (live) *reinterpret_cast<uint2*>(dst + 8 * lane_in_head) = o;
+      } else if constexpr (BITS == 4) {
+        uint32_t o = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o |= u[i] << (4 * i);
+        if (live) *reinterpret_cast<uint32_t*>(dst + 4 * lane_in_head) = o;
+      } else {
+        // 3 bits: 24 bits per lane; four neighbouring lanes make three 32-bit words
+        uint32_t o = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o |= u[i] << (3 * i);
+        const uint32_t next = __shfl_down_sync(0xffffffffu, o, 1);
+        const int r = lane_in_head & 3;
+        const uint32_t word = r == 0 ? (o | (next << 24)) : r == 1 ? ((o >> 8) | (next << 16)) : ((o >> 16) | (next << 8));
+        if (live && r < 3) *reinterpret_cast<uint32_t*>(dst + 12 * (lane_in_head >> 2) + 4 * r) = word;
+      }
+      if (live && lane_in_head == 0) scale[row] = __fdiv_rn(m, (float)(HALF - 1));
+
+      // the heads of a [BOS] token are kept at 8 bits as well
+      if (bos_codes != nullptr && live) {
+        const long token = row / n_heads;
+        if (token % seq_len == 0) {
+          const long brow = (token / seq_len) * n_heads + row % n_heads;
+          uint32_t u8[8];
+          codes8<8>(f, m, eps, u8);
+          const uint2 o = make_uint2(u8[0] | (u8[1] << 8) | (u8[2] << 16) | (u8[3] << 24), u8[4] | (u8[5] << 8) | (u8[6] << 16) | (u8[7] << 24));
+          *reinterpret_cast<uint2*>(bos_codes + brow * (8 * LPH) + 8 * lane_in_head) = o;
+          if (lane_in_head == 0) bos_scale[brow] = __fdiv_rn(m, 127.0f);
+        }
+      }
+    }
+  }
+}
+
+template <int BITS, int LPH>
+int launch_lph(const void* x, long n_rows, int n_heads, int seq_len, float eps, void* codes, float* scale, void* bos_codes,
+               float* bos_scale, cudaStream_t s) {
+  const long n_chunks = n_rows * LPH;
+  long blocks = (n_chunks + kUnroll * kThreads - 1) / (kUnroll * kThreads);
+  const long cap = (long)sm_count() * 32;                   // several waves' worth; beyond that the grid strides
+  const int grid = (int)(blocks < cap ? blocks : cap);
+  profile_before(KERNEL_ACT, s);
+  kv_quant_kernel<BITS, LPH><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(x), n_rows, n_heads, seq_len, eps,
+                                                      static_cast<unsigned char*>(codes), scale,
+                                                      static_cast<unsigned char*>(bos_codes), bos_scale);
+  profile_after(KERNEL_ACT, s);
+  note_launch();
+  HBL_CUDA_OK(cudaGetLastError());
+  return HBL_OK;
+}
+
+template <int BITS>
+int launch_bits(const void* x, long n_rows, int n_heads, int head_dim, int seq_len, float eps, void* codes, float* scale,
+                void* bos_codes, float* bos_scale, cudaStream_t s) {
+  switch (head_dim) {
+    case 64: return launch_lph<BITS, 8>(x, n_rows, n_heads, seq_len, eps, codes, scale, bos_codes, bos_scale, s);
+    case 128: return launch_lph<BITS, 16>(x, n_rows, n_heads, seq_len, eps, codes, scale, bos_codes, bos_scale, s);
+    case 256: return launch_lph<BITS, 32>(x, n_rows, n_heads, seq_len, eps, codes, scale, bos_codes, bos_scale, s);
+    default: return HBL_ERR_SHAPE;
+  }
+}
+
+}  // namespace
+
+int launch_kv_quant(const void* x, long n_rows, int n_heads, int head_dim, int bits, int seq_len, float eps, void* codes,
+                    float* scale, void* bos_codes, float* bos_scale, cudaStream_t s) {
+  if (n_rows <= 0) return HBL_OK;
+  switch (bits) {
+    case 3: return launch_bits<3>(x, n_rows, n_heads, head_dim, seq_len, eps, codes, scale, bos_codes, bos_scale, s);
+    case 4: return launch_bits<4>(x, n_rows, n_heads, head_dim, seq_len, eps, codes, scale, bos_codes, bos_scale, s);
+    case 8: return launch_bits<8>(x, n_rows, n_heads, head_dim, seq_len, eps, codes, scale, bos_codes, bos_scale, s);
+    default: return HBL_ERR_BITS;
+  }
+}
+
+}  // namespace hbl

@@ -27,7 +27,7 @@ EXPORTS = [
     "hbl_quantize_weights_workspace_bytes", "hbl_quantize_weights", "hbl_forward",
     "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_forward_glu", "hbl_glu_quantize_act", "hbl_quantize_weights_rotated", "hbl_quantize_weights_rotated_workspace_bytes",
     "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
-    "hbl_profile_events", "hbl_gemm_i32_static",
+    "hbl_profile_events", "hbl_gemm_i32_static", "hbl_kv_codes_bytes", "hbl_quantize_kv",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -83,6 +83,10 @@ def lib() -> C.CDLL:
         L.hbl_unpack_weights.argtypes = [vp, i, i, vp, vp]
         L.hbl_gemm_i32_static.argtypes = [vp, vp, i, i, vp, i, vp, vp]
         L.hbl_gemm_i32_static.restype = C.c_int
+        L.hbl_kv_codes_bytes.restype = C.c_size_t
+        L.hbl_kv_codes_bytes.argtypes = [i, i, i, i]
+        L.hbl_quantize_kv.restype = C.c_int
+        L.hbl_quantize_kv.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp, vp]
         L.hbl_forward_host.argtypes = [vp, i, i, i, vp, vp, i, i, i, f, vp, vp, vp, vp, sz, i, vp]
         L.hbl_forward_host.restype = C.c_int
         L.hbl_launch_count.restype = C.c_ulonglong
@@ -325,6 +329,25 @@ def hbl_gemm_i32_static(codes: torch.Tensor, codesum: torch.Tensor, W_packed: to
     _check(lib().hbl_gemm_i32_static(_ptr(codes), _ptr(codesum), T, K, _ptr(W_packed), out_dim, _ptr(acc),
                                      _stream()), "hbl_gemm_i32_static")
     return acc
+
+
+def hbl_quantize_kv(x: torch.Tensor, bits: int, seq_len: int = 0, eps: float = 1e-5):
+    """Section 3.1: x bf16 [tokens, n_heads, head_dim] -> (packed codes uint8 [tokens*n_heads, head_dim*bits/8],
+    scale fp32 [tokens*n_heads], bos_codes uint8 [n_seq, n_heads, head_dim] or None, bos_scale or None)."""
+    T, H, D = x.shape
+    nbytes = int(lib().hbl_kv_codes_bytes(T, H, D, bits))
+    if nbytes == 0 and T > 0:
+        raise HblError(2, "hbl_quantize_kv")
+    codes = torch.empty((T * H, D * bits // 8), dtype=torch.uint8, device=x.device)
+    scale = torch.empty((T * H,), dtype=torch.float32, device=x.device)
+    bos_codes = bos_scale = None
+    if seq_len > 0:
+        n_seq = (T + seq_len - 1) // seq_len
+        bos_codes = torch.empty((n_seq, H, D), dtype=torch.uint8, device=x.device)
+        bos_scale = torch.empty((n_seq * H,), dtype=torch.float32, device=x.device)
+    _check(lib().hbl_quantize_kv(_ptr(x), T, H, D, bits, seq_len, eps, _ptr(codes), _ptr(scale), _ptr(bos_codes),
+                                 _ptr(bos_scale), _stream()), "hbl_quantize_kv")
+    return codes, scale, bos_codes, bos_scale
 
 
 def hbl_unpack_weights(W_packed: torch.Tensor, out_dim: int, in_dim: int) -> torch.Tensor:

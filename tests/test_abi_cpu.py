@@ -85,6 +85,18 @@ def test_argument_errors_come_before_any_launch(L):
     assert L.hbl_hadamard_bf16(p, 0, 4096, p, n) == 0            # no tokens: no-op
     assert L.hbl_quantize_act(p, 0, 4, 512, 3, 1, 1e-5, p, p, p, n) == 4
     assert L.hbl_gemm_i32(p, n, 4, 512, p, 512, p, p, 1 << 30, hbl.PATH_STREAM, n) == 1   # codesum required
+    kv = lambda **kw: L.hbl_quantize_kv(kw.get("x", p), kw.get("T", 4), kw.get("H", 8), kw.get("D", 128), kw.get("bits", 4),
+                                        kw.get("S", 0), kw.get("eps", 1e-5), kw.get("codes", p), kw.get("scale", p),
+                                        kw.get("bos", n), kw.get("bos_scale", n), n)
+    assert kv(bits=5) == 4 and kv(bits=2) == 4
+    assert kv(D=96) == 2 and kv(H=0) == 2 and kv(T=-1) == 2
+    assert kv(eps=0.0) == 7
+    assert kv(bos=p, bos_scale=p, S=0) == 2                     # [BOS] rows asked for without a sequence length
+    assert kv(bos=p, S=16) == 1                                 # ... without their scales
+    assert kv(x=n) == 1 and kv(x=C.c_void_p(1032)) == 5
+    assert kv(T=0) == 0
+    L.hbl_kv_codes_bytes.restype = C.c_size_t
+    assert L.hbl_kv_codes_bytes(10, 8, 128, 3) == 10 * 8 * 48 and L.hbl_kv_codes_bytes(10, 8, 100, 4) == 0
     b = hbl.hbl_block_t()
     b.tokens, b.hidden, b.ffn, b.bits, b.x_dtype, b.eps = 4, 4096, 12288, 4, 1, 1e-5
     assert L.hbl_block_forward(C.byref(b), p, 1 << 40, 0, n) == 3                         # ffn not 2^m
