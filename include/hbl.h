@@ -200,6 +200,15 @@ int hbl_profile_events(void** start_events, void** stop_events, int n, int kerne
  * last call (HBL_OK if none) and clears it. */
 int hbl_check_status(void* stream);
 
+/* Test aid (no counterpart in the paper): makes a bounded device-side wait run out on purpose.  One small
+ * kernel waits, with a limit of limit_us microseconds (1 .. 1000000), on a barrier nobody ever arrives at, and
+ * then leaves the way every pipelined kernel of this library leaves a wait that has run out: it records
+ * HBL_ERR_TIMEOUT in the status word (hbl_check_status returns it once and clears it), raises its abort flag,
+ * a second waiting role leaves because of that flag (*left_by_abort, a device int, is then set to 1), the block
+ * drains, frees its tensor memory and returns.  Nothing traps or faults; the context stays usable.
+ * Asynchronous on `stream`. */
+int hbl_selftest_wait_timeout(int limit_us, int* left_by_abort, void* stream);
+
 /* ---- stage-level entry points (the same kernels, exposed one step at a time) ---- */
 
 /* Eq. 3-4 alone: xr_out[T,K] fp32 = H_m x, orthonormal, natural order. */

@@ -12,7 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libhbl.so")
-SOURCES = ["hbl_act.cu", "hbl_act_bf16.cu", "hbl_weights.cu", "hbl_gemm_stream.cu", "hbl_gemm_tensor.cu", "hbl_api.cu", "hbl_noalloc.cu", "hbl_kv.cu"]
+SOURCES = ["hbl_act.cu", "hbl_act_bf16.cu", "hbl_weights.cu", "hbl_gemm_stream.cu", "hbl_gemm_tensor.cu", "hbl_api.cu", "hbl_noalloc.cu", "hbl_kv.cu", "hbl_selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

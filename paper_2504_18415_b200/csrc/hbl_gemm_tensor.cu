@@ -20,10 +20,12 @@
 // returns.  No TMA multicast is used anywhere.
 #include <cuda.h>
 
-#include "hbl_common.cuh"
+#include "hbl_pipeline.cuh"
 
 namespace hbl {
 namespace {
+
+using namespace pipe;   // bounded mbarrier waits
 
 constexpr int BM = 128;              // tokens per tile (MMA M, TMEM lanes)
 constexpr int BK = 128;              // bytes (= int8 elements) of K per stage: one swizzle atom
@@ -48,10 +50,6 @@ struct Shape {
 constexpr int MAX_STAGES = 6;
 
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
 // Shared-memory matrix descriptor, K-major operand in the 128-byte swizzle:
 // start address >> 4 at [0,14); leading byte offset (unused for swizzled K-major) = 1 at [16,30);
 // stride byte offset = 1024 B between 8-row groups, >> 4, at [32,46); version 1 at [46,48);
@@ -59,48 +57,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
   return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
          (2ull << 61);
-}
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait.  Returns false when aborted (by this thread's timeout or another role's).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (mbar_try(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
-  uint32_t polls = 0;
-  while (!mbar_try(bar, parity)) {
-    if ((++polls & 255u) == 0) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > 2000000000ull) {
-        report_device_error(status, HBL_ERR_TIMEOUT);
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-  return true;
 }
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
@@ -184,7 +140,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&tfull_bar[b], 1); mbar_init(&tempty_bar[b], 4); }
     abort_flag_s = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_fence_init();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),

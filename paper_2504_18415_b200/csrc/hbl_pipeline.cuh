@@ -50,8 +50,11 @@ __device__ __forceinline__ bool mbar_try_hint(uint64_t* bar, uint32_t parity, ui
 // Returns false when aborted (this thread's timeout, or another role's).
 // POLITE waiters (anything but the thread that feeds the tensor core) park between polls so that
 // they do not take issue slots from the warps that are on the critical path.
+// limit_ns: how long the barrier may take to flip before the wait gives up (the kernels use the default).
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
 template <bool POLITE = false>
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try(bar, parity)) return true;
   if (*abort_flag) return false;
   const uint64_t t0 = global_ns();
@@ -61,7 +64,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (POLITE) __nanosleep(40);
     if ((++polls & (POLITE ? 15u : 255u)) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > 2000000000ull) {
+      if (global_ns() - t0 > limit_ns) {
         report_device_error(status, HBL_ERR_TIMEOUT);
         *abort_flag = 1;
         return false;

@@ -28,6 +28,7 @@ EXPORTS = [
     "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_forward_glu", "hbl_glu_quantize_act", "hbl_quantize_weights_rotated", "hbl_quantize_weights_rotated_workspace_bytes",
     "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
     "hbl_profile_events", "hbl_gemm_i32_static", "hbl_kv_codes_bytes", "hbl_quantize_kv",
+    "hbl_selftest_wait_timeout",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -87,6 +88,8 @@ def lib() -> C.CDLL:
         L.hbl_kv_codes_bytes.argtypes = [i, i, i, i]
         L.hbl_quantize_kv.restype = C.c_int
         L.hbl_quantize_kv.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp, vp]
+        L.hbl_selftest_wait_timeout.restype = C.c_int
+        L.hbl_selftest_wait_timeout.argtypes = [i, vp, vp]
         L.hbl_forward_host.argtypes = [vp, i, i, i, vp, vp, i, i, i, f, vp, vp, vp, vp, sz, i, vp]
         L.hbl_forward_host.restype = C.c_int
         L.hbl_launch_count.restype = C.c_ulonglong
@@ -369,6 +372,14 @@ def hbl_forward_host(x_host: torch.Tensor, W_packed: torch.Tensor, alpha: torch.
                                   _ptr(x_stage), _ptr(y_stage), _ptr(workspace), workspace.numel(), path,
                                   _stream()), "hbl_forward_host")
     return y_host
+
+
+def hbl_selftest_wait_timeout(limit_us: int = 1000) -> torch.Tensor:
+    """Launches the kernel whose bounded wait runs out (see include/hbl.h); returns the device int that the
+    second waiting role sets when it leaves because of the abort flag.  hbl_check_status() then reports the timeout."""
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().hbl_selftest_wait_timeout(limit_us, _ptr(flag), _stream()), "hbl_selftest_wait_timeout")
+    return flag
 
 
 def hbl_launch_count() -> int:
