@@ -697,6 +697,13 @@ def main():
     e2e = {"value": round(T / (e2e_ms * 1e-3), 1), "unit": "tokens/s", "h2d_bytes_per_step": T * K * 2,
            "d2h_bytes_per_step": T * N * 2, "ms_per_step": round(e2e_ms, 3), "steps": n_e2e}
 
+    # the same step with the INT4 codes kept two per byte between the two kernels (half the code traffic; the
+    # contraction widens them on the fly): reported beside the headline, which uses the faster one-per-byte form
+    def step_packed(i):
+        hbl.hbl_forward(xs[i & 1], packed, alpha, N, h["bits"], h["had"], EPS, y=ys[i & 1], workspace=work,
+                        path=hbl.PATH_TENSOR_PACKED)
+    variants = {"int4_codes_two_per_byte_ms_per_step": round(time_loop(step_packed, min(Ksteps, 10), 3, torch), 5)}
+
     ops = 2.0 * T * K * N
     ach = ops / (gemm_ms * 1e-3) / 1e12
     step_tops = ops / (ms_per_step * 1e-3) / 1e12
@@ -792,7 +799,7 @@ def main():
                    "parallelism": "replicas" if world > 1 else "single GPU"},
         "tops": round(ops / (ms_per_step * 1e-3) / 1e12, 2),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "kernels_ms": breakdown, "kernels": kernels, "roofline": roofline, "cpu_baseline": cpu, "points": points,
+        "kernels_ms": breakdown, "kernels": kernels, "variants": variants, "roofline": roofline, "cpu_baseline": cpu, "points": points,
         "peaks": {**peaks, "source": peak_src, "int8_nominal_tops": NOMINAL_INT8_TOPS, "hbm_nominal_gbs": NOMINAL_HBM_GBS,
                   **lib_i8},
     }

@@ -56,7 +56,11 @@ typedef enum { HBL_F32 = 0, HBL_BF16 = 1 } hbl_dtype_t;
 typedef enum {
   HBL_PATH_AUTO = 0,       /* by token count */
   HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers into tensor memory); tokens <= 512 */
-  HBL_PATH_TENSOR = 2      /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
+  HBL_PATH_TENSOR = 2,     /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
+  HBL_PATH_TENSOR_PACKED = 3  /* the same with the INT4 codes kept two per byte between the activation kernel and the
+                              contraction, which widens them on the fly (bits = 4, bf16 x; HBL_ERR_SHAPE where the
+                              activation kernel of the call cannot pack).  Same results, half the code traffic;
+                              measured slower than HBL_PATH_TENSOR, so HBL_PATH_AUTO never picks it */
 } hbl_path_t;
 
 const char* hbl_status_string(int status);
@@ -106,7 +110,8 @@ int hbl_quantize_weights_rotated(const void* W_latent, int w_dtype, int out_dim,
  *   bits      4 (Eq. 6) or 8 (Eq. 5);  use_hadamard: 1 applies Eq. 3-4 first
  *   y         [tokens, out_dim] bf16 (written)
  *   path      an hbl_path_t
- * The intermediate codes never leave the workspace.  On the large-batch path the
+ * The intermediate codes never leave the workspace (on the large-batch path INT4 codes are kept two per byte
+ * there, see hbl_quantize_act_int4_packed, and widened inside the contraction).  On the large-batch path the
  * packed weights are expanded to int8 (into the workspace) on a side stream of the
  * library's, which forks from `stream` at the start of the call and joins it again
  * before the contraction: in `stream`'s order the call is complete when y is.  The
@@ -238,6 +243,25 @@ int hbl_norm_quantize_act(const void* x, const void* gain, int gain_dtype, float
  * sum_k q[t,k] (may be NULL). */
 int hbl_quantize_act(const void* x, int x_dtype, int tokens, int in_dim, int bits, int use_hadamard,
                      float eps, int8_t* codes_out, float* scale_out, int32_t* codesum_out, void* stream);
+
+/* Eq. 3-4 and Eq. 6 with the quantize-AND-PACK step: INT4 codes two per byte, the form in which the large-batch
+ * path of hbl_forward / hbl_block_forward keeps them (half the bytes written by the activation kernel and read
+ * by the contraction, which widens them to int8 on the fly).
+ *   codes_packed  device, written: [tokens, in_dim / 2] bytes, 16-byte aligned.  The 32-bit little-endian word g
+ *                 of a token's row covers elements 8g .. 8g+7: byte b (0..3) of the word is
+ *                 (q[8g+b] + 8) | (q[8g+b+4] + 8) << 4, with q in [-8, 7] the code of Eq. 6.  (In this order
+ *                 `word & 0x0F0F0F0F` is four consecutive codes as bytes, `(word >> 4) & 0x0F0F0F0F` the next four.)
+ *   scale_out     device, fp32 [tokens]
+ * x must be bf16, and either use_hadamard = 1 with in_dim 2048, 4096, 8192 or 16384, or use_hadamard = 0 with
+ * more than 64 tokens (HBL_ERR_SHAPE otherwise: the other activation kernels write one code per byte).
+ * The codes are those of hbl_quantize_act(bits = 4), bit for bit. */
+int hbl_quantize_act_int4_packed(const void* x, int x_dtype, int tokens, int in_dim, int use_hadamard, float eps,
+                                 uint8_t* codes_packed, float* scale_out, void* stream);
+
+/* Eq. 7's contraction on packed INT4 codes (layout above), on the tcgen05 kernel: acc_out[T,N] int32, exact.
+ * workspace: hbl_workspace_bytes(T,K,N), 1024-byte aligned. */
+int hbl_gemm_i32_int4_packed(const uint8_t* codes_packed, int tokens, int in_dim, const void* W_packed, int out_dim,
+                             int32_t* acc_out, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Eq. 7's contraction alone: acc_out[T,N] int32 = sum_k W_t[o,k] * codes[t,k], exact.
  * codes: int8 [T,K].  codesum: int32 [T] (sum of each token's codes; required

@@ -374,7 +374,7 @@ template <int BITS>
 __global__ void __launch_bounds__(512, 2)
 quant_rows_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, int K, int NT, float eps,
                        int8_t* __restrict__ codes, float* __restrict__ scale, int32_t* __restrict__ codesum,
-                       int32_t* __restrict__ zero_fill, size_t zero_words) {
+                       int32_t* __restrict__ zero_fill, size_t zero_words, int packed) {
   __shared__ float red_f[16];
   __shared__ int red_i[16];
   grid_launch_dependents();
@@ -473,7 +473,14 @@ quant_rows_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, int K, int NT
     if (chunk < n_chunks) {
       csum = __dp4a((int)q0, 0x01010101, csum);
       csum = __dp4a((int)q1, 0x01010101, csum);
-      if (live) *reinterpret_cast<uint2*>(dst + (size_t)chunk * 8) = make_uint2(q0, q1);
+      if (BITS == 4 && packed) {
+        // INT4 codes two per byte: this chunk is the 32-bit word `chunk` of the token's K / 2 bytes,
+        // byte b = (q[b] + 8) | (q[b + 4] + 8) << 4
+        const uint32_t pk = ((q0 & 0x0F0F0F0Fu) | ((q1 & 0x0F0F0F0Fu) << 4)) ^ 0x88888888u;
+        if (live) *reinterpret_cast<uint32_t*>(codes + token * (K / 2) + (size_t)chunk * 4) = pk;
+      } else if (live) {
+        *reinterpret_cast<uint2*>(dst + (size_t)chunk * 8) = make_uint2(q0, q1);
+      }
     }
   }
 #pragma unroll
@@ -490,7 +497,7 @@ quant_rows_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, int K, int NT
 }
 
 int launch_quant_rows_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
-                           int32_t* codesum, int32_t* zf, size_t zw, cudaStream_t s) {
+                           int32_t* codesum, int32_t* zf, size_t zw, cudaStream_t s, bool packed) {
   const int n_chunks = K / 8;
   const int NT = ((n_chunks + 7) / 8 + 31) / 32 * 32;               // eight chunks per thread, whole warps
   if (NT > 512) return HBL_ERR_SHAPE;
@@ -499,10 +506,10 @@ int launch_quant_rows_bf16(const void* x, int T, int K, int bits, float eps, int
   profile_before(KERNEL_ACT, s);
   if (bits == 8)
     HBL_CUDA_OK(launch_dependent(quant_rows_bf16_kernel<8>, dim3(grid), dim3(NT * TPC), 0, s,
-                                 static_cast<const __nv_bfloat16*>(x), T, K, NT, eps, codes, scale, codesum, zf, zw));
+                                 static_cast<const __nv_bfloat16*>(x), T, K, NT, eps, codes, scale, codesum, zf, zw, (int)packed));
   else
     HBL_CUDA_OK(launch_dependent(quant_rows_bf16_kernel<4>, dim3(grid), dim3(NT * TPC), 0, s,
-                                 static_cast<const __nv_bfloat16*>(x), T, K, NT, eps, codes, scale, codesum, zf, zw));
+                                 static_cast<const __nv_bfloat16*>(x), T, K, NT, eps, codes, scale, codesum, zf, zw, (int)packed));
   profile_after(KERNEL_ACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -545,16 +552,25 @@ int dispatch(int m, const void* x, int x_dtype, int T, int bits, float eps, int8
 
 }  // namespace
 
+// Whether launch_act_quant can write INT4 codes two per byte for this call (the kernels that serve bf16 inputs
+// of more than 64 tokens can; the others write one code per byte).
+bool act_quant_can_pack(int x_dtype, int T, int K, int bits, int use_hadamard) {
+  if (bits != 4 || x_dtype != HBL_BF16) return false;
+  if (use_hadamard) return act_quant_bf16_supported(K);
+  return K % 128 == 0 && K <= 32768 && T > 64;
+}
+
 int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use_hadamard, float eps,
                      int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
-                     int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s) {
+                     int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s, bool packed) {
   if (T <= 0) return HBL_OK;
+  if (packed && (xr_out != nullptr || !act_quant_can_pack(x_dtype, T, K, bits, use_hadamard))) return HBL_ERR_SHAPE;
   if (use_hadamard && x_dtype == HBL_BF16 && act_quant_bf16_supported(K))
-    return launch_act_quant_bf16(x, T, K, bits, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s);
+    return launch_act_quant_bf16(x, T, K, bits, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, packed);
   // (a handful of tokens is a matter of latency, not bandwidth: the kernels below, with fewer elements per
   // thread, measured up to 1 us faster inside a decoder-block call of 1-16 tokens)
   if (!use_hadamard && x_dtype == HBL_BF16 && xr_out == nullptr && K % 128 == 0 && K <= 32768 && T > 64)
-    return launch_quant_rows_bf16(x, T, K, bits, eps, codes, scale, codesum, zero_fill, zero_fill_words, s);
+    return launch_quant_rows_bf16(x, T, K, bits, eps, codes, scale, codesum, zero_fill, zero_fill_words, s, packed);
   if (is_pow2(K)) {
     const int m = ilog2((unsigned)K);
     return use_hadamard

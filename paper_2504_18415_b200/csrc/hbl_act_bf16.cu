@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(Geometry<M>::THREADS, 768 / Geometry<M>::THREA
 fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
                        float* __restrict__ scale, int32_t* __restrict__ codesum, float* __restrict__ xr_out,
                        int32_t* __restrict__ zero_fill, size_t zero_words, const void* __restrict__ aux,
-                       float norm_eps) {
+                       float norm_eps, int packed) {
   using G = Geometry<M>;
   constexpr int K = G::K, NT = G::NT, THREADS = G::THREADS, TPC = G::TPC, R = G::R, C = G::C, RUN = G::RUN;
   extern __shared__ __align__(16) float smem[];
@@ -497,6 +497,24 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
   }
   __syncthreads();
 
+  if (BITS == 4 && packed) {     // uniform over the grid
+    // ---- INT4 codes two per byte: 2 chunks of 16 bytes (32 codes each) per thread.  The 32-bit word g of a
+    //      token's row covers elements 8g .. 8g+7: byte b = (q[8g+b] + 8) | (q[8g+b+4] + 8) << 4 ----
+    auto pack8 = [](uint32_t first4, uint32_t next4) {
+      return ((first4 & 0x0F0F0F0Fu) | ((next4 & 0x0F0F0F0Fu) << 4)) ^ 0x88888888u;   // q & 15 -> (q + 8) & 15
+    };
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int pc = tid + r * NT;
+      const uint4 a = *reinterpret_cast<const uint4*>(cbuf + swz_code((2 * pc) << 4));
+      const uint4 b = *reinterpret_cast<const uint4*>(cbuf + swz_code((2 * pc + 1) << 4));
+      const uint4 o = make_uint4(pack8(a.x, a.y), pack8(a.z, a.w), pack8(b.x, b.y), pack8(b.z, b.w));
+      if (live) *reinterpret_cast<uint4*>(codes + token * (K / 2) + ((size_t)pc << 4)) = o;
+    }
+    if (live && tid == 0) scale[token] = __fdiv_rn(st, cq);
+    grid_dependency_wait();
+    return;
+  }
   // ---- coalesced copy-out: 4 chunks of 16 bytes per thread ----
   int csum = 0;
 #pragma unroll
@@ -529,7 +547,7 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
 
 template <int M, int BITS, int PRE = PRE_NONE>
 int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
-               int32_t* zf, size_t zw, cudaStream_t s, const void* aux = nullptr, float norm_eps = 0.f) {
+               int32_t* zf, size_t zw, cudaStream_t s, const void* aux = nullptr, float norm_eps = 0.f, bool packed = false) {
   using G = Geometry<M>;
   const size_t smem = sizeof(float) * G::TPC * G::K;
   auto kern = fwht_quant_bf16_kernel<M, BITS, PRE>;
@@ -537,7 +555,7 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
   const int grid = (T + G::TPC - 1) / G::TPC;
   profile_before(KERNEL_ACT, s);
   HBL_CUDA_OK(launch_dependent(kern, dim3(grid), dim3(G::THREADS), smem, s, static_cast<const __nv_bfloat16*>(x), T, eps,
-                               codes, scale, codesum, xr_out, zf, zw, aux, norm_eps));
+                               codes, scale, codesum, xr_out, zf, zw, aux, norm_eps, (int)packed));
   profile_after(KERNEL_ACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -548,14 +566,14 @@ int launch_one(const void* x, int T, float eps, int8_t* codes, float* scale, int
 
 int launch_norm_act_quant_bf16(const void* x, const void* gain, int gain_dtype, float norm_eps, int T, int K, int bits,
                                float eps, int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
-                               int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s) {
+                               int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s, bool packed) {
 #define HBL_CASE(MM)                                                                                              \
   case (1 << MM):                                                                                                 \
     if (gain_dtype == HBL_BF16)                                                                                   \
-      return bits == 8 ? launch_one<MM, 8, PRE_NORM_BF16>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps) \
-                       : launch_one<MM, 4, PRE_NORM_BF16>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps); \
-    return bits == 8 ? launch_one<MM, 8, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps) \
-                     : launch_one<MM, 4, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps);
+      return bits == 8 ? launch_one<MM, 8, PRE_NORM_BF16>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps, packed) \
+                       : launch_one<MM, 4, PRE_NORM_BF16>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps, packed); \
+    return bits == 8 ? launch_one<MM, 8, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps, packed) \
+                     : launch_one<MM, 4, PRE_NORM>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, gain, norm_eps, packed);
   switch (K) {
     HBL_CASE(11) HBL_CASE(12) HBL_CASE(13) HBL_CASE(14)
     default: return HBL_ERR_SHAPE;
@@ -565,11 +583,11 @@ int launch_norm_act_quant_bf16(const void* x, const void* gain, int gain_dtype, 
 
 int launch_glu_act_quant_bf16(const void* gate, const void* up, int T, int K, int bits, float eps, int8_t* codes,
                               float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
-                              cudaStream_t s) {
+                              cudaStream_t s, bool packed) {
 #define HBL_CASE(MM)                                                                                              \
   case (1 << MM):                                                                                                 \
-    return bits == 8 ? launch_one<MM, 8, PRE_GLU>(gate, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, up, 0.f) \
-                     : launch_one<MM, 4, PRE_GLU>(gate, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, up, 0.f);
+    return bits == 8 ? launch_one<MM, 8, PRE_GLU>(gate, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, up, 0.f, packed) \
+                     : launch_one<MM, 4, PRE_GLU>(gate, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, up, 0.f, packed);
   switch (K) {
     HBL_CASE(11) HBL_CASE(12) HBL_CASE(13) HBL_CASE(14)
     default: return HBL_ERR_SHAPE;
@@ -593,11 +611,11 @@ bool act_quant_bf16_supported(int K) { return K == 2048 || K == 4096 || K == 819
 
 int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
                           int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
-                          cudaStream_t s) {
+                          cudaStream_t s, bool packed) {
 #define HBL_CASE(MM)                                                                                      \
   case (1 << MM):                                                                                         \
-    return bits == 8 ? launch_one<MM, 8>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s) \
-                     : launch_one<MM, 4>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s);
+    return bits == 8 ? launch_one<MM, 8>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, nullptr, 0.f, packed) \
+                     : launch_one<MM, 4>(x, T, eps, codes, scale, codesum, xr_out, zero_fill, zero_fill_words, s, nullptr, 0.f, packed);
   switch (K) {
     HBL_CASE(11) HBL_CASE(12) HBL_CASE(13) HBL_CASE(14)
     default: return HBL_ERR_SHAPE;

@@ -111,7 +111,7 @@ int resolve_path(int path, int tokens, size_t packed_bytes, int n_tensors) {
     return HBL_PATH_TENSOR;
   }
   if (path == HBL_PATH_STREAM) return tokens <= kStreamMaxTokens ? HBL_PATH_STREAM : -1;
-  if (path == HBL_PATH_TENSOR) return HBL_PATH_TENSOR;
+  if (path == HBL_PATH_TENSOR || path == HBL_PATH_TENSOR_PACKED) return path;
   return -2;
 }
 
@@ -152,7 +152,7 @@ int run_gemm(int path, const int8_t* codes, const float* scale, const int32_t* c
                               acc_out, acc_ws, counters, s);
   int rc = launch_unpack_weights(W_packed, N, K, w_i8, s);
   if (rc != HBL_OK) return rc;
-  return launch_gemm_tensor(codes, scale, T, K, w_i8, N, alpha, static_cast<__nv_bfloat16*>(y), acc_out, s);
+  return launch_gemm_tensor(codes, false, scale, T, K, w_i8, N, alpha, static_cast<__nv_bfloat16*>(y), acc_out, s);
 }
 
 }  // namespace
@@ -264,6 +264,11 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4, 1);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
+  // INT4 codes two per byte between the two kernels: only on request (measured slower than one code per byte
+  // at every size tried: the widening costs the contraction more than the halved code traffic saves)
+  const bool packed = (p == HBL_PATH_TENSOR_PACKED);
+  if (packed && (bits != 4 || !((gain || up) ? true : act_quant_can_pack(x_dtype, tokens > 64 ? tokens : 65, in_dim, bits, use_hadamard))))
+    return HBL_ERR_SHAPE;
   if (tokens == 0) return HBL_OK;
   if (!x || !W_packed || !alpha || !y || !workspace) return HBL_ERR_NULL;
   if (!aligned(x, 16) || !aligned(W_packed, 16) || !aligned(y, 16) || !aligned(workspace, 1024) ||
@@ -292,9 +297,9 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   int32_t* zf = stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr;
   const size_t zw = stream_path ? w.zero_words : 0;
   int32_t* cs = stream_path ? codesum : nullptr;             // only the streaming kernel needs the code sums
-  rc = gain ? launch_norm_act_quant_bf16(x, gain, gain_dtype, norm_eps, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s)
-       : up ? launch_glu_act_quant_bf16(x, up, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s)
-            : launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale, cs, nullptr, zf, zw, s);
+  rc = gain ? launch_norm_act_quant_bf16(x, gain, gain_dtype, norm_eps, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s, packed)
+       : up ? launch_glu_act_quant_bf16(x, up, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s, packed)
+            : launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale, cs, nullptr, zf, zw, s, packed);
   if (rc != HBL_OK) {
     if (sp != nullptr) cudaStreamWaitEvent(s, sp->unpacked[0], 0);   // join before reporting the error
     return rc;
@@ -304,7 +309,7 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
                               static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
                               reinterpret_cast<int*>(ws + w.counters), s);
   HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[0], 0));
-  return launch_gemm_tensor(codes, scale, tokens, in_dim, w_i8, out_dim, alpha, static_cast<__nv_bfloat16*>(y), nullptr, s);
+  return launch_gemm_tensor(codes, packed, scale, tokens, in_dim, w_i8, out_dim, alpha, static_cast<__nv_bfloat16*>(y), nullptr, s);
 }
 
 }  // namespace
@@ -423,6 +428,7 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   const int p = resolve_path(path, T, ((size_t)4 * H * H + (size_t)3 * H * F) / 4, 7);
   if (p == -1) return HBL_ERR_TOO_LARGE;
   if (p < 0) return HBL_ERR_FORMAT;
+  if (p == HBL_PATH_TENSOR_PACKED && b->bits != 4) return HBL_ERR_SHAPE;
   if (T == 0) return HBL_OK;
   const void* xs[4] = {b->x_attn_in, b->x_o_in, b->x_ffn_in, b->x_down_in};
   const void* Ws[7] = {b->Wq, b->Wk, b->Wv, b->Wo, b->Wup, b->Wgate, b->Wdown};
@@ -457,12 +463,16 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     HBL_CUDA_OK(cudaEventRecord(sp->fork, s));
     HBL_CUDA_OK(cudaStreamWaitEvent(sp->side, sp->fork, 0));
   }
+  bool packed[4] = {false, false, false, false};              // on request: INT4 codes two per byte where the kernel can
+  for (int i = 0; i < 4; ++i)
+    packed[i] = p == HBL_PATH_TENSOR_PACKED && b->bits == 4 &&
+                ((i == 3 && chain_ffn) ? true : act_quant_can_pack(b->x_dtype, T, in_dims[i], b->bits, had[i]));
   for (int i = 0; i < (chain_ffn ? 3 : 4); ++i) {
     rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
                           reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
                           stream_path ? reinterpret_cast<int32_t*>(ws + w.codesum[i]) : nullptr, nullptr,
                           (stream_path && i == 0) ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr,
-                          (stream_path && i == 0) ? w.zero_words : 0, s);
+                          (stream_path && i == 0) ? w.zero_words : 0, s, packed[i]);
     if (rc != HBL_OK) return rc;
   }
   const int src[7] = {0, 0, 0, 1, 2, 2, 3};                  // which quantized input feeds each projection
@@ -504,10 +514,10 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[i], 0));
     if (chain_ffn && i == 6) {                                // up and gate are complete in stream order
       rc = launch_glu_act_quant_bf16(ys[5], ys[4], T, F, b->bits, b->eps, reinterpret_cast<int8_t*>(ws + w.codes[3]),
-                                     reinterpret_cast<float*>(ws + w.scale[3]), nullptr, nullptr, nullptr, 0, s);
+                                     reinterpret_cast<float*>(ws + w.scale[3]), nullptr, nullptr, nullptr, 0, s, packed[3]);
       if (rc != HBL_OK) break;
     }
-    rc = launch_gemm_tensor(reinterpret_cast<int8_t*>(ws + w.codes[xi]), reinterpret_cast<float*>(ws + w.scale[xi]), T,
+    rc = launch_gemm_tensor(reinterpret_cast<int8_t*>(ws + w.codes[xi]), packed[xi], reinterpret_cast<float*>(ws + w.scale[xi]), T,
                             in_dims[xi], w_i8, out_dims[i], b->alpha7 + i, static_cast<__nv_bfloat16*>(ys[i]), nullptr, s);
     if (rc != HBL_OK) break;
     HBL_CUDA_OK(cudaEventRecord(sp->consumed[i], s));
@@ -662,6 +672,38 @@ int hbl_quantize_act(const void* x, int x_dtype, int tokens, int in_dim, int bit
                           nullptr, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
+int hbl_quantize_act_int4_packed(const void* x, int x_dtype, int tokens, int in_dim, int use_hadamard, float eps,
+                                 uint8_t* codes_packed, float* scale_out, void* stream) {
+  int rc = check_dims(tokens, in_dim, 16);
+  if (rc != HBL_OK) return rc;
+  rc = check_quant_args(x_dtype, in_dim, 4, use_hadamard, eps);
+  if (rc != HBL_OK) return rc;
+  if (!act_quant_can_pack(x_dtype, tokens > 64 ? tokens : 65, in_dim, 4, use_hadamard)) return HBL_ERR_SHAPE;
+  if (tokens == 0) return HBL_OK;
+  if (tokens <= 64 && !use_hadamard) return HBL_ERR_SHAPE;    // the small-batch kernels write one code per byte
+  if (!x || !codes_packed || !scale_out) return HBL_ERR_NULL;
+  if (!aligned(x, 16) || !aligned(codes_packed, 16) || !aligned(scale_out, 4)) return HBL_ERR_ALIGN;
+  return launch_act_quant(x, x_dtype, tokens, in_dim, 4, use_hadamard, eps, reinterpret_cast<int8_t*>(codes_packed), scale_out,
+                          nullptr, nullptr, nullptr, 0, static_cast<cudaStream_t>(stream), true);
+}
+
+int hbl_gemm_i32_int4_packed(const uint8_t* codes_packed, int tokens, int in_dim, const void* W_packed, int out_dim,
+                             int32_t* acc_out, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_dims(tokens, in_dim, out_dim);
+  if (rc != HBL_OK) return rc;
+  if (tokens == 0) return HBL_OK;
+  if (!codes_packed || !W_packed || !acc_out || !workspace) return HBL_ERR_NULL;
+  if (!aligned(codes_packed, 16) || !aligned(W_packed, 16) || !aligned(acc_out, 16) || !aligned(workspace, 1024))
+    return HBL_ERR_ALIGN;
+  const ForwardWs w = carve(tokens, in_dim, out_dim);
+  if (workspace_bytes < w.total) return HBL_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int8_t* w_i8 = reinterpret_cast<int8_t*>(static_cast<char*>(workspace) + w.w_i8);
+  rc = launch_unpack_weights(W_packed, out_dim, in_dim, w_i8, s);
+  if (rc != HBL_OK) return rc;
+  return launch_gemm_tensor(codes_packed, true, nullptr, tokens, in_dim, w_i8, out_dim, nullptr, nullptr, acc_out, s);
+}
+
 int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in_dim, const void* W_packed,
                  int out_dim, int32_t* acc_out, void* workspace, size_t workspace_bytes, int path, void* stream) {
   int rc = check_dims(tokens, in_dim, out_dim);
@@ -671,6 +713,7 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
   if (p < 0) return HBL_ERR_FORMAT;
   if (tokens == 0) return HBL_OK;
   if (!codes || !W_packed || !acc_out || !workspace) return HBL_ERR_NULL;
+  if (p == HBL_PATH_TENSOR_PACKED) return HBL_ERR_FORMAT;      // these codes are one per byte: see hbl_gemm_i32_int4_packed
   if (p == HBL_PATH_STREAM && !codesum) return HBL_ERR_NULL;
   if (!aligned(codes, 16) || !aligned(W_packed, 16) || !aligned(acc_out, 16) || !aligned(workspace, 1024))
     return HBL_ERR_ALIGN;

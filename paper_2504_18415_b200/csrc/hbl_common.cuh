@@ -81,22 +81,25 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 
 // ---- kernel launchers (one per .cu file) -------------------------------------
 // Activation side: Eq. 3-6.
+// packed: INT4 codes are written two per byte ([T, K / 2] bytes, layout in hbl.h) instead of one; only where
+// act_quant_can_pack() says so (HBL_ERR_SHAPE otherwise), and never together with codesum or xr_out.
+bool act_quant_can_pack(int x_dtype, int T, int K, int bits, int use_hadamard);
 int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use_hadamard, float eps,
                      int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
-                     int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s);
+                     int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s, bool packed = false);
 // The same for bf16 inputs with the transform on (tensor-core first stages, packed fp32 butterflies).
 bool act_quant_bf16_supported(int K);
 int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
                           int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
-                          cudaStream_t s);
+                          cudaStream_t s, bool packed = false);
 // The same with the token RMS-normalised and multiplied by gain[K] (fp32 or bf16, device) first ("LN" of Eq. 7).
 int launch_norm_act_quant_bf16(const void* x, const void* gain, int gain_dtype, float norm_eps, int T, int K, int bits,
                                float eps, int8_t* codes, float* scale, int32_t* codesum, float* xr_out,
-                               int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s);
+                               int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s, bool packed = false);
 // The same with the token replaced by SiLU(gate) * up first (both bf16 [T, K]): the SwishGLU input of W_down.
 int launch_glu_act_quant_bf16(const void* gate, const void* up, int T, int K, int bits, float eps, int8_t* codes,
                               float* scale, int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
-                              cudaStream_t s);
+                              cudaStream_t s, bool packed = false);
 // The transform alone, bf16 in and out (Eq. 8: the backward pass applies it to the gradient); K as above.
 int launch_hadamard_bf16(const void* x, int T, int K, void* out, cudaStream_t s);
 // Weight side: Eq. 1-2 and the 2-bit format.
@@ -116,7 +119,8 @@ struct GemmSegment {          // one weight tensor of a (possibly fused) project
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
                        const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s);
-int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
+// codes: int8 [T, K], or (codes_packed) INT4 codes two per byte [T, K / 2] in the layout hbl.h gives.
+int launch_gemm_tensor(const void* codes, bool codes_packed, const float* scale, int T, int K, const int8_t* W_i8, int N,
                        const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s);
 // Several weight tensors, each reading one of up to four quantized inputs, per launch; one launch per 128 tokens.
 int gemm_stream_max_tokens();

@@ -35,11 +35,18 @@ constexpr int THREADS = 192;
 constexpr int TMEM_COLS = 512;
 // Weight rows per tile (MMA N, TMEM columns): 256 is the efficient shape; 128 is used when 256-row tiles
 // would leave half of the SMs without a tile (it doubles the number of tiles).
-template <int BN>
+// PACKED: the tokens' INT4 codes arrive two per byte (Eq. 6's codes, packed by the activation kernel).  Each
+// stage then also holds the 8 KiB packed tile as TMA delivers it, and eight more warps widen it into the int8
+// token tile the tensor cores read.
+constexpr int PK_BYTES = BM * BK / 2;                    // packed token tile of one stage: 128 rows x 64 bytes
+constexpr int WIDEN_THREADS = 256;                       // two threads per token row of the tile
+template <int BN, bool PACKED = false>
 struct Shape {
-  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int STAGES = BN == 256 ? 4 : (PACKED ? 5 : 6);
   static constexpr int B_BYTES = BN * BK;                // 32 or 16 KiB
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TX_BYTES = (PACKED ? PK_BYTES : A_BYTES) + B_BYTES;     // what the copies of one stage deliver
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + (PACKED ? PK_BYTES : 0);
+  static constexpr int N_THREADS = THREADS + (PACKED ? WIDEN_THREADS : 0);
   static constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024;   // + alignment slack
   // Instruction descriptor (32 bit): D format s32 (2) at bits [4,6); A and B format
   // signed 8-bit (1) at [7,10) and [10,13); both K-major (bits 15, 16 = 0);
@@ -114,15 +121,16 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
   n0 = (local / gm) * BN;
 }
 
-template <int BN>
-__global__ void __launch_bounds__(THREADS, 1)
+template <int BN, bool PACKED>
+__global__ void __launch_bounds__(Shape<BN, PACKED>::N_THREADS, 1)
 gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const float* __restrict__ scale, const float* __restrict__ alpha,
                    __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out, int T, int N, int K,
                    int* __restrict__ status) {
-  constexpr int STAGES = Shape<BN>::STAGES, STAGE_BYTES = Shape<BN>::STAGE_BYTES;
+  constexpr int STAGES = Shape<BN, PACKED>::STAGES, STAGE_BYTES = Shape<BN, PACKED>::STAGE_BYTES;
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t wide_bar[MAX_STAGES];    // PACKED: the stage's token tile has been widened
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t tfull_bar[2];
   __shared__ __align__(8) uint64_t tempty_bar[2];
@@ -137,7 +145,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   const int nkb = K / BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); mbar_init(&wide_bar[s], WIDEN_THREADS / 32); }
     for (int b = 0; b < 2; ++b) { mbar_init(&tfull_bar[b], 1); mbar_init(&tempty_bar[b], 4); }
     abort_flag_s = 0;
     mbar_fence_init();
@@ -163,9 +171,10 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1, abort_flag, status)) { ok = false; break; }
-          mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+          mbar_expect_tx(&full_bar[s], Shape<BN, PACKED>::TX_BYTES);
           unsigned char* a = tiles + (size_t)s * STAGE_BYTES;
-          tma_load_2d(a, &tmA, &full_bar[s], kb * BK, m0);
+          if constexpr (PACKED) tma_load_2d(a + A_BYTES + Shape<BN, PACKED>::B_BYTES, &tmA, &full_bar[s], kb * (BK / 2), m0);
+          else tma_load_2d(a, &tmA, &full_bar[s], kb * BK, m0);
           tma_load_2d(a + A_BYTES, &tmB, &full_bar[s], kb * BK, n0);
         }
       }
@@ -182,17 +191,62 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         const uint32_t d_tmem = tmem_base + (uint32_t)b * BN;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGES;
-          if (!mbar_wait(&full_bar[s], (it / STAGES) & 1, abort_flag, status)) { ok = false; break; }
+          // (the widen warps waited for the stage's copies before they wrote the token tile: one wait covers both)
+          if (!mbar_wait(PACKED ? &wide_bar[s] : &full_bar[s], (it / STAGES) & 1, abort_flag, status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(tiles + (size_t)s * STAGE_BYTES);
           const uint64_t adesc = make_desc(a_addr), bdesc = make_desc(a_addr + A_BYTES);
 #pragma unroll
           for (int ks = 0; ks < BK / UMMA_K; ++ks)
             umma_i8(d_tmem, adesc + (uint64_t)(ks * UMMA_K / 16), bdesc + (uint64_t)(ks * UMMA_K / 16),
-                    Shape<BN>::IDESC, (kb | ks) != 0);
+                    Shape<BN, PACKED>::IDESC, (kb | ks) != 0);
           umma_commit(&empty_bar[s]);          // stage reusable once these MMAs have read it
         }
         if (ok) umma_commit(&tfull_bar[b]);    // accumulator complete
+      }
+    }
+  } else if (warp >= THREADS / 32) {
+    // ------------------------------ widen (PACKED only) ------------------------------
+    // Two threads own token row r of the tile, two 16-byte pieces (32 codes) of its 64 packed bytes each.  The
+    // 32-bit word g of a packed row covers elements 8g .. 8g+7, byte b = (q[8g+b] + 8) | (q[8g+b+4] + 8) << 4:
+    // `w & 0x0F0F0F0F` is four consecutive codes (plus 8) as bytes, `(w >> 4) & 0x0F0F0F0F` the next four, and a
+    // per-byte subtraction of 8 makes them the signed int8 values the MMA reads.  They are written where a
+    // 128-byte-swizzled TMA load would have put them: row r at r * 128, its 16-byte chunk c at position c ^ (r & 7).
+    if constexpr (PACKED) {
+      const int r = ((int)threadIdx.x - THREADS) & (BM - 1);
+      const int half = ((int)threadIdx.x - THREADS) >> 7;
+      auto widen = [](const uint4& w, uint4& lo, uint4& hi) {
+        lo.x = __vsub4(w.x & 0x0F0F0F0Fu, 0x08080808u); lo.y = __vsub4((w.x >> 4) & 0x0F0F0F0Fu, 0x08080808u);
+        lo.z = __vsub4(w.y & 0x0F0F0F0Fu, 0x08080808u); lo.w = __vsub4((w.y >> 4) & 0x0F0F0F0Fu, 0x08080808u);
+        hi.x = __vsub4(w.z & 0x0F0F0F0Fu, 0x08080808u); hi.y = __vsub4((w.z >> 4) & 0x0F0F0F0Fu, 0x08080808u);
+        hi.z = __vsub4(w.w & 0x0F0F0F0Fu, 0x08080808u); hi.w = __vsub4((w.w >> 4) & 0x0F0F0F0Fu, 0x08080808u);
+      };
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          ok = __all_sync(0xffffffffu, mbar_wait<true>(&full_bar[s], (it / STAGES) & 1, abort_flag, status));
+          if (!ok) break;
+          unsigned char* stage = tiles + (size_t)s * STAGE_BYTES;
+          const unsigned char* pk = stage + A_BYTES + Shape<BN, PACKED>::B_BYTES + r * (BK / 2);
+          unsigned char* row = stage + r * BK;
+#pragma unroll
+          for (int j = 2 * half; j < 2 * half + 2; ++j) {
+            // piece order j ^ g(r), g = 0, 2, 3, 1 for (r >> 1) & 3 = 0..3: with it the eight threads of a
+            // quarter-warp hit distinct banks both in the loads (row pitch 64 bytes) and in the swizzled stores
+            const int jj = j ^ ((0x78 >> (r & 6)) & 3);
+            const uint4 w = *reinterpret_cast<const uint4*>(pk + 16 * jj);
+            uint4 lo, hi;
+            widen(w, lo, hi);
+            *reinterpret_cast<uint4*>(row + 16 * ((2 * jj) ^ (r & 7))) = lo;
+            *reinterpret_cast<uint4*>(row + 16 * ((2 * jj + 1) ^ (r & 7))) = hi;
+          }
+          // generic-proxy writes, read next by the tensor cores (async proxy)
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&wide_bar[s]);
+        }
       }
     }
   } else {
@@ -290,21 +344,38 @@ int make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) 
   return r == CUDA_SUCCESS ? HBL_OK : HBL_ERR_CUDA;
 }
 
-template <int BN>
-int launch_shape(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N, const float* alpha,
+// Packed INT4 codes [rows, K / 2] bytes row-major, box = 128 rows x 64 bytes, no swizzle (the widen warps read it
+// row by row), zero fill.
+int make_map_packed(CUtensorMap* map, const void* base, int rows, int K) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return HBL_ERR_CUDA;
+  cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+  cuuint32_t box[2] = {(cuuint32_t)(BK / 2), (cuuint32_t)BM};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? HBL_OK : HBL_ERR_CUDA;
+}
+
+template <int BN, bool PACKED>
+int launch_shape(const void* codes, const float* scale, int T, int K, const int8_t* W_i8, int N, const float* alpha,
                  __nv_bfloat16* y, int32_t* acc_out, int n_sm, cudaStream_t s) {
   CUtensorMap tmA, tmB;
-  int rc = make_map(&tmA, codes, T, K, BM);
+  int rc = PACKED ? make_map_packed(&tmA, codes, T, K) : make_map(&tmA, codes, T, K, BM);
   if (rc != HBL_OK) return rc;
   rc = make_map(&tmB, W_i8, N, K, BN);
   if (rc != HBL_OK) return rc;
-  HBL_ALLOW_DYNAMIC_SMEM(gemm_tensor_kernel<BN>, Shape<BN>::SMEM_BYTES);
+  auto kern = gemm_tensor_kernel<BN, PACKED>;
+  using SH = Shape<BN, PACKED>;
+  HBL_ALLOW_DYNAMIC_SMEM(kern, SH::SMEM_BYTES);
   int* status = device_status_word();
   if (status == nullptr) return HBL_ERR_CUDA;
   const int n_tiles = ((T + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
   profile_before(KERNEL_CONTRACT, s);
-  gemm_tensor_kernel<BN><<<grid, THREADS, Shape<BN>::SMEM_BYTES, s>>>(tmA, tmB, scale, alpha, y, acc_out, T, N, K, status);
+  kern<<<grid, SH::N_THREADS, SH::SMEM_BYTES, s>>>(tmA, tmB, scale, alpha, y, acc_out, T, N, K, status);
   profile_after(KERNEL_CONTRACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -313,7 +384,7 @@ int launch_shape(const int8_t* codes, const float* scale, int T, int K, const in
 
 }  // namespace
 
-int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, const int8_t* W_i8, int N,
+int launch_gemm_tensor(const void* codes, bool codes_packed, const float* scale, int T, int K, const int8_t* W_i8, int N,
                        const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s) {
   if (T <= 0) return HBL_OK;
   const int n_sm = sm_count();
@@ -323,8 +394,13 @@ int launch_gemm_tensor(const int8_t* codes, const float* scale, int T, int K, co
   // larger sizes small-batch contractions are bound by L2 traffic, which narrower tiles increase
   // (8192 -> 2048 at 1024 tokens: 37.6 -> 39.2 us; a 7B block at 4096 tokens: 0.96 -> 1.13 ms).
   const long t128 = (long)((T + BM - 1) / BM) * ((N + 127) / 128);
-  if (N > 128 && 2 * t128 <= n_sm) return launch_shape<128>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
-  return launch_shape<256>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
+  const bool narrow = N > 128 && 2 * t128 <= n_sm;
+  if (codes_packed) {
+    if (narrow) return launch_shape<128, true>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
+    return launch_shape<256, true>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
+  }
+  if (narrow) return launch_shape<128, false>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
+  return launch_shape<256, false>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
 }
 
 }  // namespace hbl

@@ -14,7 +14,7 @@ import torch
 
 HBL_OK = 0
 HBL_F32, HBL_BF16 = 0, 1
-PATH_AUTO, PATH_STREAM, PATH_TENSOR = 0, 1, 2
+PATH_AUTO, PATH_STREAM, PATH_TENSOR, PATH_TENSOR_PACKED = 0, 1, 2, 3
 
 STATUS_NAMES = {
     0: "HBL_OK", 1: "HBL_ERR_NULL", 2: "HBL_ERR_SHAPE", 3: "HBL_ERR_NOT_POW2", 4: "HBL_ERR_BITS",
@@ -28,7 +28,7 @@ EXPORTS = [
     "hbl_block_workspace_bytes", "hbl_block_forward", "hbl_check_status", "hbl_hadamard_f32", "hbl_hadamard_bf16", "hbl_forward_norm", "hbl_norm_quantize_act", "hbl_forward_glu", "hbl_glu_quantize_act", "hbl_quantize_weights_rotated", "hbl_quantize_weights_rotated_workspace_bytes",
     "hbl_quantize_act", "hbl_gemm_i32", "hbl_unpack_weights", "hbl_forward_host", "hbl_launch_count",
     "hbl_profile_events", "hbl_gemm_i32_static", "hbl_kv_codes_bytes", "hbl_quantize_kv",
-    "hbl_selftest_wait_timeout",
+    "hbl_selftest_wait_timeout", "hbl_quantize_act_int4_packed", "hbl_gemm_i32_int4_packed",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -88,6 +88,10 @@ def lib() -> C.CDLL:
         L.hbl_kv_codes_bytes.argtypes = [i, i, i, i]
         L.hbl_quantize_kv.restype = C.c_int
         L.hbl_quantize_kv.argtypes = [vp, i, i, i, i, i, f, vp, vp, vp, vp, vp]
+        L.hbl_quantize_act_int4_packed.restype = C.c_int
+        L.hbl_quantize_act_int4_packed.argtypes = [vp, i, i, i, i, f, vp, vp, vp]
+        L.hbl_gemm_i32_int4_packed.restype = C.c_int
+        L.hbl_gemm_i32_int4_packed.argtypes = [vp, i, i, vp, i, vp, vp, sz, vp]
         L.hbl_selftest_wait_timeout.restype = C.c_int
         L.hbl_selftest_wait_timeout.argtypes = [i, vp, vp]
         L.hbl_forward_host.argtypes = [vp, i, i, i, vp, vp, i, i, i, f, vp, vp, vp, vp, sz, i, vp]
@@ -310,6 +314,27 @@ def hbl_quantize_act(x: torch.Tensor, bits: int, use_hadamard: bool, eps: float 
     _check(lib().hbl_quantize_act(_ptr(x), _dt(x), T, K, bits, int(bool(use_hadamard)), eps, _ptr(codes),
                                   _ptr(scale), _ptr(csum), _stream()), "hbl_quantize_act")
     return codes, scale, csum
+
+
+def hbl_quantize_act_int4_packed(x: torch.Tensor, use_hadamard: bool, eps: float = 1e-5):
+    """Eq. 3-4, 6 with the pack step: returns (codes uint8 [T, K/2], two INT4 codes per byte, scale fp32 [T])."""
+    T, K = x.shape
+    codes = torch.empty((T, K // 2), dtype=torch.uint8, device=x.device)
+    scale = torch.empty((T,), dtype=torch.float32, device=x.device)
+    _check(lib().hbl_quantize_act_int4_packed(_ptr(x), _dt(x), T, K, int(bool(use_hadamard)), eps, _ptr(codes), _ptr(scale),
+                                              _stream()), "hbl_quantize_act_int4_packed")
+    return codes, scale
+
+
+def hbl_gemm_i32_int4_packed(codes_packed: torch.Tensor, W_packed: torch.Tensor, out_dim: int,
+                             workspace: torch.Tensor | None = None) -> torch.Tensor:
+    T, K = codes_packed.shape[0], codes_packed.shape[1] * 2
+    acc = torch.empty((T, out_dim), dtype=torch.int32, device=codes_packed.device)
+    if workspace is None:
+        workspace = new_workspace(hbl_workspace_bytes(T, K, out_dim), codes_packed.device)
+    _check(lib().hbl_gemm_i32_int4_packed(_ptr(codes_packed), T, K, _ptr(W_packed), out_dim, _ptr(acc), _ptr(workspace),
+                                          workspace.numel(), _stream()), "hbl_gemm_i32_int4_packed")
+    return acc
 
 
 def hbl_gemm_i32(codes: torch.Tensor, codesum: torch.Tensor | None, W_packed: torch.Tensor, out_dim: int,
