@@ -528,6 +528,16 @@ def block_point(T, torch, hbl, peaks, iters=None):
 HEAD = dict(name="config3_Wdown_1p3B", kind="ffn_mid", seed=3, K=8192, N=2048, bits=4, had=True, T=16384)
 
 
+def headline_config(world: int) -> dict:
+    """The `config` object of the JSON line: the same in both arms (the reference arm times a bounded sample of it)."""
+    h = HEAD
+    return {"workload": f"{h['name']}: H-BitLinear in 8192 -> out 2048, INT4 activations + Hadamard, "
+                        f"{h['T']} tokens per step, bf16 activations SiLU(a)*b with 0.2% outlier channels x40, "
+                        f"ternary weights from N(0,0.02) latents",
+            "l2": "two alternating 268 MB input batches (each larger than the 126 MB L2)",
+            "parallelism": "replicas" if world > 1 else "single GPU"}
+
+
 def oracle_rate(target_s=12.0):
     """Times the oracle as it stands on a bounded token sample of the headline workload."""
     from oracle import hbl_oracle as orc
@@ -574,8 +584,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": round(val, 2), "unit": UNIT,
         "n_gpus": args.gpus, "steps": steps, "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{HEAD['name']}: in 8192 -> out 2048, INT4 + Hadamard, bf16 activations (SiLU(a)*b with "
-                               f"0.2% outlier channels x40), {HEAD['T']} tokens per step on the GPU arm; bounded sample here"},
+        "config": headline_config(int(os.environ.get("WORLD_SIZE", "1"))),
         "cpu_baseline": {"value": round(val, 2), "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": round(val, 2), "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -699,9 +708,14 @@ def main():
 
     # the same step with the INT4 codes kept two per byte between the two kernels (half the code traffic; the
     # contraction widens them on the fly): reported beside the headline, which uses the faster one-per-byte form
-    def step_packed(i):
+    pk_state = {"i": 0}
+
+    def step_packed():
+        i = pk_state["i"]
+        pk_state["i"] += 1
         hbl.hbl_forward(xs[i & 1], packed, alpha, N, h["bits"], h["had"], EPS, y=ys[i & 1], workspace=work,
                         path=hbl.PATH_TENSOR_PACKED)
+
     variants = {"int4_codes_two_per_byte_ms_per_step": round(time_loop(step_packed, min(Ksteps, 10), 3, torch), 5)}
 
     ops = 2.0 * T * K * N
@@ -792,11 +806,7 @@ def main():
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": Ksteps, "warmup": W,
         "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "s8", "data": "synthetic",
-        "config": {"workload": f"{h['name']}: H-BitLinear in 8192 -> out 2048, INT4 activations + Hadamard, "
-                               f"{T} tokens per step, bf16 activations SiLU(a)*b with 0.2% outlier channels x40, "
-                               f"ternary weights from N(0,0.02) latents",
-                   "l2": "two alternating 268 MB input batches (each larger than the 126 MB L2)",
-                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "config": headline_config(world),
         "tops": round(ops / (ms_per_step * 1e-3) / 1e12, 2),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "kernels_ms": breakdown, "kernels": kernels, "variants": variants, "roofline": roofline, "cpu_baseline": cpu, "points": points,

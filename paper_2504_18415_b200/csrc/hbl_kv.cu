@@ -19,19 +19,21 @@ constexpr int kThreads = 256;
 constexpr int kUnroll = 4;                                   // 16-byte chunks in flight per thread
 constexpr float kMagic = 12582912.0f;                        // 1.5 * 2^23: x + kMagic has rint(x) in its low mantissa bits
 
-// Codes of 8 consecutive elements for width BITS, from the fp32 values f and the head's maximum g.
-// IEEE fp32, operations in the order the formula is written: c / (g + eps), times x, round to nearest even, clip.
-// (Clipping to the integer bounds first and rounding by the magic-number add gives the same integers as
-// rounding first: the bounds are integers and |v| is far below 2^22.)
+// Codes of 8 consecutive elements for width BITS, from the fp32 values f and the head's maximum g, as the low
+// bytes of u[0..7].  IEEE fp32, operations in the order the formula is written: c / (g + eps), times x, round to
+// nearest even.  No clip is needed: |x| <= g gives |v| <= c g / (g + eps) < c = 2^(BITS-1) - 1, so the rounded
+// value already lies inside [-2^(BITS-1), 2^(BITS-1) - 1].  The rounding is the magic-number add (|v| is far
+// below 2^22), with the offset 2^(BITS-1) folded into the constant: the low byte of the sum is the unsigned code.
 template <int BITS>
 __device__ __forceinline__ void codes8(const float (&f)[8], float g, float eps, uint32_t (&u)[8]) {
   constexpr int HALF = 1 << (BITS - 1);
   const float rq = __fdiv_rn((float)(HALF - 1), __fadd_rn(g, eps));
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const float v = fminf(fmaxf(__fmul_rn(rq, f[i]), (float)-HALF), (float)(HALF - 1));
-    u[i] = (__float_as_uint(__fadd_rn(v, kMagic + (float)HALF))) & 0xFFu;      // rint(v) + HALF, in [0, 2 HALF - 1]
-  }
+  for (int i = 0; i < 8; ++i) u[i] = __float_as_uint(__fadd_rn(__fmul_rn(rq, f[i]), kMagic + (float)HALF));
+}
+// The low bytes of four words as one word (byte i = low byte of u[i]).
+__device__ __forceinline__ uint32_t low_bytes(uint32_t u0, uint32_t u1, uint32_t u2, uint32_t u3) {
+  return __byte_perm(__byte_perm(u0, u1, 0x0040), __byte_perm(u2, u3, 0x0040), 0x5410);
 }
 
 // LPH = lanes per head = head_dim / 8.  A thread block takes tiles of kUnroll x kThreads chunks; a thread's
@@ -60,32 +62,34 @@ kv_quant_kernel(const uint4* __restrict__ x, long n_rows, int n_heads, int seq_l
       const long row = (live ? chunk : n_chunks - 1) / LPH;
       const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
       float f[8];
-      float m = 0.f;
+      uint32_t m2 = 0;                                        // a pair of bf16 maxima of |x|
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         f[2 * i] = __uint_as_float(w[i] << 16);
         f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-        m = fmaxf(m, fmaxf(fabsf(f[2 * i]), fabsf(f[2 * i + 1])));
+        const uint32_t a = w[i] & 0x7FFF7FFFu;
+        const __nv_bfloat162 h = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&m2), *reinterpret_cast<const __nv_bfloat162*>(&a));
+        m2 = *reinterpret_cast<const uint32_t*>(&h);
       }
+      float m = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
 #pragma unroll
       for (int o = LPH / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
 
       uint32_t u[8];
       codes8<BITS>(f, m, eps, u);
+      const uint32_t b0 = low_bytes(u[0], u[1], u[2], u[3]), b1 = low_bytes(u[4], u[5], u[6], u[7]);   // codes as bytes
       unsigned char* dst = codes + row * ROW_BYTES;
       if constexpr (BITS == 8) {
-        const uint2 o = make_uint2(u[0] | (u[1] << 8) | (u[2] << 16) | (u[3] << 24), u[4] | (u[5] << 8) | (u[6] << 16) | (u[7] << 24));
-        if (live) *reinterpret_cast<uint2*>(dst + 8 * lane_in_head) = o;
+        if (live) *reinterpret_cast<uint2*>(dst + 8 * lane_in_head) = make_uint2(b0, b1);
       } else if constexpr (BITS == 4) {
-        uint32_t o = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o |= u[i] << (4 * i);
+        // byte pairs to nibble pairs: (x | x >> 4) has code 0 | code 1 << 4 in byte 0 and code 2 | code 3 << 4 in byte 2
+        const uint32_t o = __byte_perm(b0 | (b0 >> 4), b1 | (b1 >> 4), 0x6420);
         if (live) *reinterpret_cast<uint32_t*>(dst + 4 * lane_in_head) = o;
       } else {
         // 3 bits: 24 bits per lane; four neighbouring lanes make three 32-bit words
         uint32_t o = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) o |= u[i] << (3 * i);
+        for (int i = 0; i < 4; ++i) o |= (((b0 >> (8 * i)) & 7u) << (3 * i)) | (((b1 >> (8 * i)) & 7u) << (3 * i + 12));
         const uint32_t next = __shfl_down_sync(0xffffffffu, o, 1);
         const int r = lane_in_head & 3;
         const uint32_t word = r == 0 ? (o | (next << 24)) : r == 1 ? ((o >> 8) | (next << 16)) : ((o >> 16) | (next << 8));
@@ -100,7 +104,7 @@ kv_quant_kernel(const uint4* __restrict__ x, long n_rows, int n_heads, int seq_l
           const long brow = (token / seq_len) * n_heads + row % n_heads;
           uint32_t u8[8];
           codes8<8>(f, m, eps, u8);
-          const uint2 o = make_uint2(u8[0] | (u8[1] << 8) | (u8[2] << 16) | (u8[3] << 24), u8[4] | (u8[5] << 8) | (u8[6] << 16) | (u8[7] << 24));
+          const uint2 o = make_uint2(low_bytes(u8[0], u8[1], u8[2], u8[3]), low_bytes(u8[4], u8[5], u8[6], u8[7]));
           *reinterpret_cast<uint2*>(bos_codes + brow * (8 * LPH) + 8 * lane_in_head) = o;
           if (lane_in_head == 0) bos_scale[brow] = __fdiv_rn(m, 127.0f);
         }
