@@ -19,15 +19,14 @@ constexpr int kThreads = 256;
 constexpr int kUnroll = 4;                                   // 16-byte chunks in flight per thread
 constexpr float kMagic = 12582912.0f;                        // 1.5 * 2^23: x + kMagic has rint(x) in its low mantissa bits
 
-// Codes of 8 consecutive elements for width BITS, from the fp32 values f and the head's maximum g, as the low
-// bytes of u[0..7].  IEEE fp32, operations in the order the formula is written: c / (g + eps), times x, round to
-// nearest even.  No clip is needed: |x| <= g gives |v| <= c g / (g + eps) < c = 2^(BITS-1) - 1, so the rounded
-// value already lies inside [-2^(BITS-1), 2^(BITS-1) - 1].  The rounding is the magic-number add (|v| is far
-// below 2^22), with the offset 2^(BITS-1) folded into the constant: the low byte of the sum is the unsigned code.
+// Codes of 8 consecutive elements for width BITS, as the low bytes of u[0..7], from the fp32 values f and the
+// head's factor rq = c / (gamma + eps), c = 2^(BITS-1) - 1: IEEE fp32 product, round to nearest even.  No clip
+// is needed: |x| <= gamma gives |v| <= c gamma / (gamma + eps) < c, so the rounded value already lies inside
+// [-2^(BITS-1), 2^(BITS-1) - 1].  The rounding is the magic-number add (|v| is far below 2^22), with the offset
+// 2^(BITS-1) folded into the constant: the low byte of the sum is the unsigned code.
 template <int BITS>
-__device__ __forceinline__ void codes8(const float (&f)[8], float g, float eps, uint32_t (&u)[8]) {
+__device__ __forceinline__ void codes8(const float (&f)[8], float rq, uint32_t (&u)[8]) {
   constexpr int HALF = 1 << (BITS - 1);
-  const float rq = __fdiv_rn((float)(HALF - 1), __fadd_rn(g, eps));
 #pragma unroll
   for (int i = 0; i < 8; ++i) u[i] = __float_as_uint(__fadd_rn(__fmul_rn(rq, f[i]), kMagic + (float)HALF));
 }
@@ -35,9 +34,20 @@ __device__ __forceinline__ void codes8(const float (&f)[8], float g, float eps, 
 __device__ __forceinline__ uint32_t low_bytes(uint32_t u0, uint32_t u1, uint32_t u2, uint32_t u3) {
   return __byte_perm(__byte_perm(u0, u1, 0x0040), __byte_perm(u2, u3, 0x0040), 0x5410);
 }
+__device__ __forceinline__ void widen8(const uint4& raw, float (&f)[8]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
 
 // LPH = lanes per head = head_dim / 8.  A thread block takes tiles of kUnroll x kThreads chunks; a thread's
-// kUnroll loads are issued before any arithmetic.
+// kUnroll loads are issued before any arithmetic.  The two IEEE divisions of a head (c / (gamma + eps) and
+// gamma / c) are what costs most instructions here, and a warp pays for a division whatever the number of its
+// lanes that need it: so the maxima of all heads a warp holds in a tile (kUnroll x 32 / LPH of them) are
+// gathered one per lane, divided once, and the factors handed back by shuffles.
 template <int BITS, int LPH>
 __global__ void __launch_bounds__(kThreads)
 kv_quant_kernel(const uint4* __restrict__ x, long n_rows, int n_heads, int seq_len, float eps,
@@ -46,37 +56,57 @@ kv_quant_kernel(const uint4* __restrict__ x, long n_rows, int n_heads, int seq_l
   constexpr int HALF = 1 << (BITS - 1);
   constexpr int ROW_BYTES = LPH * BITS;                     // head_dim * BITS / 8
   constexpr long TILE = (long)kUnroll * kThreads;
+  constexpr int HPW = 32 / LPH;                             // heads a warp holds per chunk row
   const long n_chunks = n_rows * LPH;                       // (a multiple of LPH: a head is live or dead as a whole)
-  const int lane_in_head = threadIdx.x % LPH;
+  const int lane = threadIdx.x & 31;
+  const int lane_in_head = lane % LPH;
   for (long tile0 = (long)blockIdx.x * TILE; tile0 < n_chunks; tile0 += (long)gridDim.x * TILE) {
     uint4 raw[kUnroll];
+    float m[kUnroll];
 #pragma unroll
     for (int k = 0; k < kUnroll; ++k) {
       const long chunk = tile0 + k * kThreads + threadIdx.x;
       raw[k] = chunk < n_chunks ? __ldg(x + chunk) : make_uint4(0, 0, 0, 0);
     }
+    // ---- per-head maximum of |x| (on bf16 pairs), shared by the head's lanes ----
+#pragma unroll
+    for (int k = 0; k < kUnroll; ++k) {
+      const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+      uint32_t m2 = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t a = w[i] & 0x7FFF7FFFu;
+        const __nv_bfloat162 h = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&m2), *reinterpret_cast<const __nv_bfloat162*>(&a));
+        m2 = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      float v = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
+#pragma unroll
+      for (int o = LPH / 2; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      m[k] = v;
+    }
+    // ---- lane j < kUnroll * HPW takes head (k = j / HPW, h = j % HPW): both divisions, and the scale store ----
+    float g = 0.f;
+#pragma unroll
+    for (int k = 0; k < kUnroll; ++k) {
+      const float t = __shfl_sync(0xffffffffu, m[k], (lane % HPW) * LPH);
+      if (lane / HPW == k) g = t;
+    }
+    const float rq_mine = __fdiv_rn((float)(HALF - 1), __fadd_rn(g, eps));
+    if (lane < kUnroll * HPW) {
+      const long chunk = tile0 + (lane / HPW) * kThreads + (threadIdx.x & ~31) + (lane % HPW) * LPH;
+      if (chunk < n_chunks) scale[chunk / LPH] = __fdiv_rn(g, (float)(HALF - 1));
+    }
+    // ---- quantize and pack ----
 #pragma unroll
     for (int k = 0; k < kUnroll; ++k) {
       const long chunk = tile0 + k * kThreads + threadIdx.x;
       const bool live = chunk < n_chunks;
       const long row = (live ? chunk : n_chunks - 1) / LPH;
-      const uint32_t w[4] = {raw[k].x, raw[k].y, raw[k].z, raw[k].w};
+      const float rq = __shfl_sync(0xffffffffu, rq_mine, k * HPW + lane / LPH);
       float f[8];
-      uint32_t m2 = 0;                                        // a pair of bf16 maxima of |x|
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        f[2 * i] = __uint_as_float(w[i] << 16);
-        f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-        const uint32_t a = w[i] & 0x7FFF7FFFu;
-        const __nv_bfloat162 h = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&m2), *reinterpret_cast<const __nv_bfloat162*>(&a));
-        m2 = *reinterpret_cast<const uint32_t*>(&h);
-      }
-      float m = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xFFFF0000u));
-#pragma unroll
-      for (int o = LPH / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-
+      widen8(raw[k], f);
       uint32_t u[8];
-      codes8<BITS>(f, m, eps, u);
+      codes8<BITS>(f, rq, u);
       const uint32_t b0 = low_bytes(u[0], u[1], u[2], u[3]), b1 = low_bytes(u[4], u[5], u[6], u[7]);   // codes as bytes
       unsigned char* dst = codes + row * ROW_BYTES;
       if constexpr (BITS == 8) {
@@ -95,18 +125,16 @@ kv_quant_kernel(const uint4* __restrict__ x, long n_rows, int n_heads, int seq_l
         const uint32_t word = r == 0 ? (o | (next << 24)) : r == 1 ? ((o >> 8) | (next << 16)) : ((o >> 16) | (next << 8));
         if (live && r < 3) *reinterpret_cast<uint32_t*>(dst + 12 * (lane_in_head >> 2) + 4 * r) = word;
       }
-      if (live && lane_in_head == 0) scale[row] = __fdiv_rn(m, (float)(HALF - 1));
-
       // the heads of a [BOS] token are kept at 8 bits as well
       if (bos_codes != nullptr && live) {
         const long token = row / n_heads;
         if (token % seq_len == 0) {
           const long brow = (token / seq_len) * n_heads + row % n_heads;
           uint32_t u8[8];
-          codes8<8>(f, m, eps, u8);
+          codes8<8>(f, __fdiv_rn(127.0f, __fadd_rn(m[k], eps)), u8);
           const uint2 o = make_uint2(low_bytes(u8[0], u8[1], u8[2], u8[3]), low_bytes(u8[4], u8[5], u8[6], u8[7]));
           *reinterpret_cast<uint2*>(bos_codes + brow * (8 * LPH) + 8 * lane_in_head) = o;
-          if (lane_in_head == 0) bos_scale[brow] = __fdiv_rn(m, 127.0f);
+          if (lane_in_head == 0) bos_scale[brow] = __fdiv_rn(m[k], 127.0f);
         }
       }
     }
