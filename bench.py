@@ -44,9 +44,9 @@ METRIC = "H-BitLinear tokens/s and TOPS vs INT8 tensor peak; HBM GB/s at small b
 UNIT = "tokens/s"
 ALU_PEAK_LANE_OPS = 148 * 128 * 1.965e9      # fp32 lanes x SMs x clocks.max.sm
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dominant kernel at the headline workload, copied
-# from an ncu capture of that kernel (156.23 MB read + 49.68 MB written); a constant, not re-measured by a run.
+# from an ncu capture of that kernel (151.78 MB read + 48.57 MB written); a constant, not re-measured by a run.
 # None whenever the kernel has changed since the counters were taken.
-GEMM_TENSOR_TRAFFIC_BYTES = 205914112
+GEMM_TENSOR_TRAFFIC_BYTES = 200351744
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
