@@ -119,6 +119,18 @@ struct GemmSegment {          // one weight tensor of a (possibly fused) project
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
                        const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
                        int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s);
+// Several weight tensors that read the same quantized input (q | k | v, up | gate), contracted as ONE matrix of
+// concatenated weight rows: output i takes the rows [begin[i], begin[i] + width[i]) of W_i8, has its own alpha
+// and its own bf16 tensor [T, width[i]].  begin[0] = 0, the widths of all but the last are multiples of 256.
+constexpr int kMaxTensorOutputs = 3;
+struct TensorOutputs {
+  int n;
+  int begin[kMaxTensorOutputs], width[kMaxTensorOutputs];
+  __nv_bfloat16* y[kMaxTensorOutputs];
+  const float* alpha[kMaxTensorOutputs];
+};
+int launch_gemm_tensor_multi(const void* codes, bool codes_packed, const float* scale, int T, int K, const int8_t* W_i8,
+                             const TensorOutputs& outs, int32_t* acc_out, cudaStream_t s);
 // codes: int8 [T, K], or (codes_packed) INT4 codes two per byte [T, K / 2] in the layout hbl.h gives.
 int launch_gemm_tensor(const void* codes, bool codes_packed, const float* scale, int T, int K, const int8_t* W_i8, int N,
                        const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s);

@@ -124,8 +124,8 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 template <int BN, bool PACKED>
 __global__ void __launch_bounds__(Shape<BN, PACKED>::N_THREADS, 1)
 gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                   const float* __restrict__ scale, const float* __restrict__ alpha,
-                   __nv_bfloat16* __restrict__ y, int32_t* __restrict__ acc_out, int T, int N, int K,
+                   const float* __restrict__ scale, const __grid_constant__ TensorOutputs outs,
+                   int32_t* __restrict__ acc_out, int T, int N, int K,
                    int* __restrict__ status) {
   constexpr int STAGES = Shape<BN, PACKED>::STAGES, STAGE_BYTES = Shape<BN, PACKED>::STAGE_BYTES;
   extern __shared__ unsigned char smem_dyn[];
@@ -252,7 +252,6 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   } else {
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;                    // TMEM lane quadrant this warp may access
-    const float al = (acc_out == nullptr) ? __ldg(alpha) : 0.f;
     uint32_t tl = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tl) {
       const int b = tl & 1;
@@ -262,13 +261,18 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       if (!__all_sync(0xffffffffu, got)) break;      // warp-uniform: tcgen05.ld needs the whole warp
       tc_fence_after();
       const int row = m0 + q * 32 + lane;
-      const float f = (acc_out == nullptr && row < T) ? __ldg(scale + row) * al : 0.f;
+      // the weight rows of this tile belong to one output tensor (segments start on tile boundaries)
+      int si = 0;
+      while (si + 1 < outs.n && n0 >= outs.begin[si + 1]) ++si;
+      const int seg_n0 = n0 - outs.begin[si], seg_N = (acc_out != nullptr) ? N : outs.width[si];
+      __nv_bfloat16* __restrict__ y = outs.y[si];
+      const float f = (acc_out == nullptr && row < T) ? __ldg(scale + row) * __ldg(outs.alpha[si]) : 0.f;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c * 32), r);
         tmem_ld_wait();
-        const int col = n0 + c * 32;
+        const int col = seg_n0 + c * 32;
         if (row < T) {
           if (acc_out != nullptr) {
             int32_t* dst = acc_out + (size_t)row * N + col;
@@ -276,10 +280,10 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             for (int i = 0; i < 32; i += 4)
               if (col + i < N) *reinterpret_cast<uint4*>(dst + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
           } else {
-            __nv_bfloat16* dst = y + (size_t)row * N + col;
+            __nv_bfloat16* dst = y + (size_t)row * seg_N + col;
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
-              if (col + i < N) {
+              if (col + i < seg_N) {
                 uint4 o;
                 o.x = pack_bf16((float)(int)r[i + 0] * f, (float)(int)r[i + 1] * f);
                 o.y = pack_bf16((float)(int)r[i + 2] * f, (float)(int)r[i + 3] * f);
@@ -360,8 +364,8 @@ int make_map_packed(CUtensorMap* map, const void* base, int rows, int K) {
 }
 
 template <int BN, bool PACKED>
-int launch_shape(const void* codes, const float* scale, int T, int K, const int8_t* W_i8, int N, const float* alpha,
-                 __nv_bfloat16* y, int32_t* acc_out, int n_sm, cudaStream_t s) {
+int launch_shape(const void* codes, const float* scale, int T, int K, const int8_t* W_i8, int N, const TensorOutputs& outs,
+                 int32_t* acc_out, int n_sm, cudaStream_t s) {
   CUtensorMap tmA, tmB;
   int rc = PACKED ? make_map_packed(&tmA, codes, T, K) : make_map(&tmA, codes, T, K, BM);
   if (rc != HBL_OK) return rc;
@@ -375,7 +379,7 @@ int launch_shape(const void* codes, const float* scale, int T, int K, const int8
   const int n_tiles = ((T + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
   profile_before(KERNEL_CONTRACT, s);
-  kern<<<grid, SH::N_THREADS, SH::SMEM_BYTES, s>>>(tmA, tmB, scale, alpha, y, acc_out, T, N, K, status);
+  kern<<<grid, SH::N_THREADS, SH::SMEM_BYTES, s>>>(tmA, tmB, scale, outs, acc_out, T, N, K, status);
   profile_after(KERNEL_CONTRACT, s);
   note_launch();
   HBL_CUDA_OK(cudaGetLastError());
@@ -384,9 +388,16 @@ int launch_shape(const void* codes, const float* scale, int T, int K, const int8
 
 }  // namespace
 
-int launch_gemm_tensor(const void* codes, bool codes_packed, const float* scale, int T, int K, const int8_t* W_i8, int N,
-                       const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s) {
+int launch_gemm_tensor_multi(const void* codes, bool codes_packed, const float* scale, int T, int K, const int8_t* W_i8,
+                             const TensorOutputs& outs, int32_t* acc_out, cudaStream_t s) {
   if (T <= 0) return HBL_OK;
+  if (outs.n < 1 || outs.n > kMaxTensorOutputs) return HBL_ERR_SHAPE;
+  int N = 0;
+  for (int i = 0; i < outs.n; ++i) {
+    if (outs.begin[i] != N || outs.width[i] <= 0) return HBL_ERR_SHAPE;
+    if (i + 1 < outs.n && outs.width[i] % 256 != 0) return HBL_ERR_SHAPE;    // a tile never straddles two outputs
+    N += outs.width[i];
+  }
   const int n_sm = sm_count();
   // The narrow tile only pays on very small grids, where even twice as many tiles leave half of the SMs
   // idle (measured: 2048 x 2048 at 256 tokens 14.3 -> 12.8 us).  It costs about 1.5x per weight row (a
@@ -396,11 +407,18 @@ int launch_gemm_tensor(const void* codes, bool codes_packed, const float* scale,
   const long t128 = (long)((T + BM - 1) / BM) * ((N + 127) / 128);
   const bool narrow = N > 128 && 2 * t128 <= n_sm;
   if (codes_packed) {
-    if (narrow) return launch_shape<128, true>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
-    return launch_shape<256, true>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
+    if (narrow) return launch_shape<128, true>(codes, scale, T, K, W_i8, N, outs, acc_out, n_sm, s);
+    return launch_shape<256, true>(codes, scale, T, K, W_i8, N, outs, acc_out, n_sm, s);
   }
-  if (narrow) return launch_shape<128, false>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
-  return launch_shape<256, false>(codes, scale, T, K, W_i8, N, alpha, y, acc_out, n_sm, s);
+  if (narrow) return launch_shape<128, false>(codes, scale, T, K, W_i8, N, outs, acc_out, n_sm, s);
+  return launch_shape<256, false>(codes, scale, T, K, W_i8, N, outs, acc_out, n_sm, s);
+}
+
+int launch_gemm_tensor(const void* codes, bool codes_packed, const float* scale, int T, int K, const int8_t* W_i8, int N,
+                       const float* alpha, __nv_bfloat16* y, int32_t* acc_out, cudaStream_t s) {
+  TensorOutputs outs = {};
+  outs.n = 1; outs.begin[0] = 0; outs.width[0] = N; outs.y[0] = y; outs.alpha[0] = alpha;
+  return launch_gemm_tensor_multi(codes, codes_packed, scale, T, K, W_i8, outs, acc_out, s);
 }
 
 }  // namespace hbl

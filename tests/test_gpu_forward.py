@@ -165,3 +165,29 @@ def test_forward_host_equals_forward(T):
         torch.cuda.current_stream().synchronize()      # the caller's stream alone: it waits for the side streams
         assert hbl.hbl_check_status() == 0
         assert torch.equal(yh, want)
+
+
+def test_block_large_batch_equals_seven_separate_layers():
+    """On the large-batch path q | k | v and up | gate are contracted as one matrix each (one launch, per-output alpha
+    and output tensor).  The integers and the rounding are those of seven separate hbl_forward calls: bit-equal."""
+    H, F, T = 1024, 4096, 700                                   # (fused up to 2048 tokens)
+    seed = 35
+    ins_np = {"attn_in": wl.rows("gauss", seed, 10, H, 0, T, "bf16"), "o_in": wl.rows("attn_out", seed, 11, H, 0, T, "bf16"),
+              "ffn_in": wl.rows("gauss", seed, 12, H, 0, T, "bf16"), "down_in": wl.rows("ffn_mid", seed, 13, F, 0, T, "bf16")}
+    ins = {k: to_dev(v, "bf16") for k, v in ins_np.items()}
+    shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "up": (F, H), "gate": (F, H), "down": (H, F)}
+    src = {"q": "attn_in", "k": "attn_in", "v": "attn_in", "o": "o_in", "up": "ffn_in", "gate": "ffn_in", "down": "down_in"}
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    packed, alphas = {}, []
+    for n, (N, K) in shapes.items():
+        p, a = hbl.hbl_quantize_weights(torch.randn((N, K), device="cuda", generator=g) * 0.02, EPS)
+        packed[n] = p; alphas.append(a)
+    outs = hbl.hbl_block_forward(ins, packed, torch.cat(alphas), H, F, 4, EPS, path=hbl.PATH_TENSOR)
+    assert hbl.hbl_check_status() == 0
+    for i, (n, (N, K)) in enumerate(shapes.items()):
+        y = hbl.hbl_forward(ins[src[n]], packed[n], alphas[i], N, 4, n in ("o", "down"), EPS, path=hbl.PATH_TENSOR)
+        assert torch.equal(outs[n], y), n
+    # called again on the same workspace-free path the result repeats (buffers of the int8 weights are reused)
+    again = hbl.hbl_block_forward(ins, packed, torch.cat(alphas), H, F, 4, EPS, path=hbl.PATH_TENSOR)
+    for n in shapes:
+        assert torch.equal(again[n], outs[n]), n
