@@ -22,6 +22,7 @@
 //   * Codes are assembled in shared memory (over the exchange buffer, which is
 //     dead by then) and leave with coalesced 128-bit stores.
 #include "hbl_common.cuh"
+#include "hbl_quant_rows.cuh"
 
 namespace hbl {
 namespace {
@@ -99,11 +100,11 @@ __device__ __forceinline__ int swz_word(int a) { return a ^ ((((a >> 5) ^ (a >> 
 // Byte address swizzle of the code staging area (keeps 16-byte chunks intact).
 __device__ __forceinline__ int swz_code(int i) { return i ^ (((i >> 9) & 3) << 5); }
 
-template <int M>
+template <int M, int MIN_THREADS = 128>
 struct Geometry {
   static constexpr int K = 1 << M;
   static constexpr int NT = K / 64;                       // threads per token
-  static constexpr int THREADS = NT < 128 ? 128 : NT;
+  static constexpr int THREADS = NT < MIN_THREADS ? MIN_THREADS : NT;
   static constexpr int TPC = THREADS / NT;                // tokens per CTA
   static constexpr int R = M - 8;                         // index bits [5, 5+R) are transformed in the final phase
   static constexpr int C = 6 - R;                         // low bits kept thread-local for contiguity
@@ -145,31 +146,22 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int group, in
 //   PRE_GLU   the SwishGLU product that feeds W_down: x' = bf16(SiLU(x) * aux), aux = the other projection's
 //             output, bf16 [T, K] (x is the one that passes through SiLU).
 enum { PRE_NONE = 0, PRE_NORM = 1, PRE_GLU = 2, PRE_NORM_BF16 = 3 };   // PRE_NORM_BF16: the same with a bf16 gain
-template <int M, int BITS, int PRE = PRE_NONE>
-__global__ void __launch_bounds__(Geometry<M>::THREADS, 768 / Geometry<M>::THREADS)
-fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
-                       float* __restrict__ scale, int32_t* __restrict__ codesum, float* __restrict__ xr_out,
-                       int32_t* __restrict__ zero_fill, size_t zero_words, const void* __restrict__ aux,
-                       float norm_eps, int packed) {
-  using G = Geometry<M>;
-  constexpr int K = G::K, NT = G::NT, THREADS = G::THREADS, TPC = G::TPC, R = G::R, C = G::C, RUN = G::RUN;
-  extern __shared__ __align__(16) float smem[];
-  __shared__ float red_f[THREADS / 32];
-  __shared__ int red_i[THREADS / 32];
-
-  // A kernel launched as a programmatic dependent of this one may start now; it waits
-  // (griddepcontrol.wait) before it touches anything written here.
-  grid_launch_dependents();
+// The body serves the tokens block * TPC ... of one input with a thread block of Geometry<M, MIN_THREADS>::THREADS
+// threads: `smem` is TPC * K floats of shared memory aligned to 128 bytes (the swizzles toggle address
+// bits up to 6), `red_f` / `red_i` are THREADS / 32 words each.
+template <int M, int BITS, int PRE = PRE_NONE, int MIN_THREADS = 128>
+__device__ __forceinline__ void fwht_quant_body(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
+                                                float* __restrict__ scale, int32_t* __restrict__ codesum,
+                                                float* __restrict__ xr_out, const void* __restrict__ aux, float norm_eps,
+                                                int packed, long block, float* smem, float* red_f, int* red_i) {
+  using G = Geometry<M, MIN_THREADS>;
+  constexpr int K = G::K, NT = G::NT, TPC = G::TPC, R = G::R, C = G::C, RUN = G::RUN;
   const int tid_cta = threadIdx.x;
-  if (zero_fill != nullptr) {   // side job: clear the caller's scratch words
-    for (size_t i = (size_t)blockIdx.x * THREADS + tid_cta; i < zero_words; i += (size_t)gridDim.x * THREADS)
-      zero_fill[i] = 0;
-  }
   const int group = tid_cta / NT;
   const int tid = tid_cta % NT;
   const int lane = tid_cta & 31, warp_cta = tid_cta >> 5;
   const int warp = tid >> 5;                               // warp inside the token group
-  const long token_raw = (long)blockIdx.x * TPC + group;
+  const long token_raw = block * TPC + group;
   const bool live = token_raw < T;
   const long token = live ? token_raw : (long)T - 1;       // a dead group recomputes the last token, stores nothing
   float* buf = smem + (size_t)group * K;
@@ -405,7 +397,6 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
         }
       }
     }
-    grid_dependency_wait();
     return;
   }
   if (xr_out != nullptr) {       // stage export (uniform over the grid): x_r in fp32, nothing else
@@ -512,7 +503,6 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
       if (live) *reinterpret_cast<uint4*>(codes + token * (K / 2) + ((size_t)pc << 4)) = o;
     }
     if (live && tid == 0) scale[token] = __fdiv_rn(st, cq);
-    grid_dependency_wait();
     return;
   }
   // ---- coalesced copy-out: 4 chunks of 16 bytes per thread ----
@@ -542,6 +532,27 @@ fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, in
     if (live && tid == 0) codesum[token] = csum;
   }
   if (live && tid == 0) scale[token] = __fdiv_rn(st, cq);
+}
+
+template <int M, int BITS, int PRE = PRE_NONE>
+__global__ void __launch_bounds__(Geometry<M>::THREADS, 768 / Geometry<M>::THREADS)
+fwht_quant_bf16_kernel(const __nv_bfloat16* __restrict__ x, int T, float eps, int8_t* __restrict__ codes,
+                       float* __restrict__ scale, int32_t* __restrict__ codesum, float* __restrict__ xr_out,
+                       int32_t* __restrict__ zero_fill, size_t zero_words, const void* __restrict__ aux,
+                       float norm_eps, int packed) {
+  constexpr int THREADS = Geometry<M>::THREADS;
+  extern __shared__ __align__(128) float smem[];
+  __shared__ float red_f[THREADS / 32];
+  __shared__ int red_i[THREADS / 32];
+  // A kernel launched as a programmatic dependent of this one may start now; it waits (griddepcontrol.wait)
+  // before it touches anything written here.
+  grid_launch_dependents();
+  if (zero_fill != nullptr) {   // side job: clear the caller's scratch words
+    for (size_t i = (size_t)blockIdx.x * THREADS + threadIdx.x; i < zero_words; i += (size_t)gridDim.x * THREADS)
+      zero_fill[i] = 0;
+  }
+  fwht_quant_body<M, BITS, PRE>(x, T, eps, codes, scale, codesum, xr_out, aux, norm_eps, packed, (long)blockIdx.x, smem,
+                                red_f, red_i);
   grid_dependency_wait();   // chain: this kernel is complete only when the one before it is
 }
 
@@ -621,6 +632,112 @@ int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8
     default: return HBL_ERR_SHAPE;
   }
 #undef HBL_CASE
+}
+
+// ---- several bf16 inputs of the same token count in one launch ----
+// A decoder block quantizes four inputs before its contraction.  As four kernels they are four dependent
+// launches, each a microsecond or two of latency that a handful of tokens cannot hide; here every input gets a
+// range of thread blocks of one grid.  Inputs with the transform run fwht_quant_body (K = 2^11..2^14), inputs
+// without it quant_rows_bf16_body (K a multiple of 128, at most 16384), all with 256 threads per block.
+namespace {
+
+constexpr int kMultiThreads = 256;
+constexpr size_t kMultiMaxSmem = sizeof(float) * 16384;
+
+struct ActMultiParams {
+  ActJob job[kMaxActJobs];
+  int first_block[kMaxActJobs + 1];   // input j owns blocks [first_block[j], first_block[j + 1])
+  int nt[kMaxActJobs];                // threads per token of an input without the transform
+  int n, T;
+  float eps;
+  int32_t* zero_fill;
+  size_t zero_words;
+};
+
+template <int BITS>
+__global__ void __launch_bounds__(kMultiThreads)
+act_multi_bf16_kernel(const __grid_constant__ ActMultiParams p) {
+  extern __shared__ __align__(128) float smem[];
+  __shared__ float red_f[16];
+  __shared__ int red_i[16];
+  grid_launch_dependents();   // the contraction that follows may start and fetch its first weights
+  if (p.zero_fill != nullptr)
+    for (size_t i = (size_t)blockIdx.x * kMultiThreads + threadIdx.x; i < p.zero_words; i += (size_t)gridDim.x * kMultiThreads)
+      p.zero_fill[i] = 0;
+  int j = 0;
+  while (j + 1 < p.n && (int)blockIdx.x >= p.first_block[j + 1]) ++j;
+  const ActJob& job = p.job[j];
+  const long block = (long)blockIdx.x - p.first_block[j];
+  const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(job.x);
+  if (!job.use_hadamard) {
+    quant_rows_bf16_body<BITS>(x, p.T, job.K, p.nt[j], p.eps, job.codes, job.scale, job.codesum, 0, block, red_f, red_i);
+    grid_dependency_wait();   // chain: this kernel is complete only when the one before it is
+    return;
+  }
+#define HBL_CASE(MM)                                                                                                \
+  case (1 << MM):                                                                                                   \
+    fwht_quant_body<MM, BITS, PRE_NONE, kMultiThreads>(x, p.T, p.eps, job.codes, job.scale, job.codesum, nullptr, nullptr, \
+                                                       0.f, 0, block, smem, red_f, red_i);                          \
+    break;
+  switch (job.K) {
+    HBL_CASE(11) HBL_CASE(12) HBL_CASE(13) HBL_CASE(14)
+    default: break;
+  }
+#undef HBL_CASE
+  grid_dependency_wait();
+}
+
+}  // namespace
+
+bool act_multi_bf16_supported(const ActJob* jobs, int n_jobs) {
+  if (n_jobs < 1 || n_jobs > kMaxActJobs) return false;
+  for (int j = 0; j < n_jobs; ++j) {
+    const int K = jobs[j].K;
+    if (jobs[j].use_hadamard ? !act_quant_bf16_supported(K) : (K % 128 != 0 || K > 16384)) return false;
+  }
+  return true;
+}
+
+int launch_act_multi_bf16(const ActJob* jobs, int n_jobs, int T, int bits, float eps, int32_t* zero_fill,
+                          size_t zero_fill_words, cudaStream_t s) {
+  if (T <= 0) return HBL_OK;
+  if (!act_multi_bf16_supported(jobs, n_jobs)) return HBL_ERR_SHAPE;
+  if (bits != 4 && bits != 8) return HBL_ERR_BITS;
+  ActMultiParams p{};
+  size_t smem = 0;
+  int blocks = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    p.job[j] = jobs[j];
+    p.first_block[j] = blocks;
+    const int K = jobs[j].K;
+    int tpc;
+    if (jobs[j].use_hadamard) {
+      const int nt = K / 64;
+      tpc = nt < kMultiThreads ? kMultiThreads / nt : 1;
+      const size_t need = sizeof(float) * (size_t)tpc * K;
+      if (need > smem) smem = need;
+    } else {
+      p.nt[j] = ((K / 8 + 7) / 8 + 31) / 32 * 32;           // eight 16-byte chunks per thread, whole warps
+      tpc = kMultiThreads / p.nt[j];
+    }
+    blocks += (T + tpc - 1) / tpc;
+  }
+  p.first_block[n_jobs] = blocks;
+  p.n = n_jobs;
+  p.T = T;
+  p.eps = eps;
+  p.zero_fill = zero_fill;
+  p.zero_words = zero_fill_words;
+  auto kern = bits == 8 ? act_multi_bf16_kernel<8> : act_multi_bf16_kernel<4>;
+  // (the attribute is set once per device, to the most any supported input needs: 2^14 floats)
+  if (bits == 8) HBL_ALLOW_DYNAMIC_SMEM(act_multi_bf16_kernel<8>, kMultiMaxSmem);
+  else HBL_ALLOW_DYNAMIC_SMEM(act_multi_bf16_kernel<4>, kMultiMaxSmem);
+  profile_before(KERNEL_ACT, s);
+  HBL_CUDA_OK(launch_dependent(kern, dim3(blocks), dim3(kMultiThreads), smem, s, p));
+  profile_after(KERNEL_ACT, s);
+  note_launch();
+  HBL_CUDA_OK(cudaGetLastError());
+  return HBL_OK;
 }
 
 }  // namespace hbl

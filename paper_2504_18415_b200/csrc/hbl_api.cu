@@ -468,7 +468,23 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   for (int i = 0; i < 4; ++i)
     packed[i] = p == HBL_PATH_TENSOR_PACKED && b->bits == 4 &&
                 ((i == 3 && chain_ffn) ? true : act_quant_can_pack(b->x_dtype, T, in_dims[i], b->bits, had[i]));
-  for (int i = 0; i < (chain_ffn ? 3 : 4); ++i) {
+  // small batch, bf16 inputs: one launch quantizes all inputs (each launch is a dependent step of a microsecond
+  // or two, which is what a call of a few tokens spends most of its time on besides the weights)
+  const int n_act = chain_ffn ? 3 : 4;
+  bool one_launch = false;
+  if (stream_path && b->x_dtype == HBL_BF16) {
+    ActJob aj[4];
+    for (int i = 0; i < n_act; ++i)
+      aj[i] = {xs[i], reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
+               reinterpret_cast<int32_t*>(ws + w.codesum[i]), in_dims[i], had[i]};
+    if (act_multi_bf16_supported(aj, n_act)) {
+      rc = launch_act_multi_bf16(aj, n_act, T, b->bits, b->eps, reinterpret_cast<int32_t*>(ws + w.zero_region),
+                                 w.zero_words, s);
+      if (rc != HBL_OK) return rc;
+      one_launch = true;
+    }
+  }
+  for (int i = 0; i < (one_launch ? 0 : n_act); ++i) {
     rc = launch_act_quant(xs[i], b->x_dtype, T, in_dims[i], b->bits, had[i], b->eps,
                           reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
                           stream_path ? reinterpret_cast<int32_t*>(ws + w.codesum[i]) : nullptr, nullptr,

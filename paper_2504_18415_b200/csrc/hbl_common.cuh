@@ -89,6 +89,12 @@ int launch_act_quant(const void* x, int x_dtype, int T, int K, int bits, int use
                      int32_t* zero_fill, size_t zero_fill_words, cudaStream_t s, bool packed = false);
 // The same for bf16 inputs with the transform on (tensor-core first stages, packed fp32 butterflies).
 bool act_quant_bf16_supported(int K);
+// Several bf16 inputs of T tokens each, quantized by one launch (Eq. 3-6 per input).
+constexpr int kMaxActJobs = 4;
+struct ActJob { const void* x; int8_t* codes; float* scale; int32_t* codesum; int K; int use_hadamard; };
+bool act_multi_bf16_supported(const ActJob* jobs, int n_jobs);
+int launch_act_multi_bf16(const ActJob* jobs, int n_jobs, int T, int bits, float eps, int32_t* zero_fill,
+                          size_t zero_fill_words, cudaStream_t s);
 int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
                           int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
                           cudaStream_t s, bool packed = false);

@@ -101,6 +101,37 @@ def test_block_forward_small():
             check_y(outs[n], o["y64"])
 
 
+@pytest.mark.parametrize("H,F,bits,T", [(2048, 8192, 8, 3), (2048, 8192, 4, 70), (4096, 8192, 4, 17), (2048, 16384, 8, 130)])
+def test_block_small_batch_one_launch_quantizer(H, F, bits, T):
+    """Small batches of bf16 inputs: one launch quantizes the four inputs of the block (transform sizes 2^11..2^14
+    mixed with inputs that skip the transform).  Against the oracle, and bit for bit against the large-batch
+    launch configuration, which quantizes each input with a kernel of its own."""
+    seed = 47
+    ins = {"attn_in": wl.rows("gauss", seed, 10, H, 0, T, "bf16"), "o_in": wl.rows("attn_out", seed, 11, H, 0, T, "bf16"),
+           "ffn_in": wl.rows("gauss", seed, 12, H, 0, T, "bf16"), "down_in": wl.rows("ffn_mid", seed, 13, F, 0, T, "bf16")}
+    shapes = {"q": (H, H), "k": (H, H), "v": (H, H), "o": (H, H), "up": (F, H), "gate": (F, H), "down": (H, F)}
+    src = {"q": "attn_in", "k": "attn_in", "v": "attn_in", "o": "o_in", "up": "ffn_in", "gate": "ffn_in", "down": "down_in"}
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    packed, alphas, Wl = {}, [], {}
+    for n, (N, K) in shapes.items():
+        W = torch.randn((N, K), device="cuda", generator=g) * 0.02
+        p, a = hbl.hbl_quantize_weights(W, EPS)
+        packed[n] = p; alphas.append(a)
+        Wl[n] = W.cpu().numpy()
+    alpha7 = torch.cat(alphas)
+    dev = {k: to_dev(v, "bf16") for k, v in ins.items()}
+    outs = hbl.hbl_block_forward(dev, packed, alpha7, H, F, bits, EPS, path=hbl.PATH_STREAM)
+    assert hbl.hbl_check_status() == 0
+    outs = {n: v.clone() for n, v in outs.items()}
+    ref = hbl.hbl_block_forward(dev, packed, alpha7, H, F, bits, EPS, path=hbl.PATH_TENSOR)
+    assert hbl.hbl_check_status() == 0
+    for n in shapes:
+        assert torch.equal(outs[n], ref[n]), f"{n}: the two launch configurations differ"
+    for n in ("q", "o", "gate", "down"):
+        o = oracle_layer(ins[src[n]], Wl[n], bits, n in ("o", "down"))
+        check_y(outs[n], o["y64"])
+
+
 def test_zero_tokens_is_a_noop():
     packed, alpha = hbl.hbl_quantize_weights(torch.zeros((16, 128), device="cuda"), EPS)
     y = hbl.hbl_forward(torch.empty((0, 128), dtype=torch.bfloat16, device="cuda"), packed, alpha, 16, 4, True)
