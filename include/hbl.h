@@ -57,10 +57,21 @@ typedef enum {
   HBL_PATH_AUTO = 0,       /* by token count */
   HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers into tensor memory); tokens <= 512 */
   HBL_PATH_TENSOR = 2,     /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
-  HBL_PATH_TENSOR_PACKED = 3  /* the same with the INT4 codes kept two per byte between the activation kernel and the
+  HBL_PATH_TENSOR_PACKED = 3, /* the same with the INT4 codes kept two per byte between the activation kernel and the
                               contraction, which widens them on the fly (bits = 4, bf16 x; HBL_ERR_SHAPE where the
                               activation kernel of the call cannot pack).  Same results, half the code traffic;
                               measured slower than HBL_PATH_TENSOR, so HBL_PATH_AUTO never picks it */
+  HBL_PATH_STREAM_OVERLAP = 4 /* HBL_PATH_STREAM for calls issued back to back on one stream with no other work between
+                              them (hbl_forward and hbl_block_forward): the contraction releases its programmatic
+                              dependents as soon as it has seen its quantizer complete, so the next such call's
+                              quantizer runs beside it and the next contraction takes over the SMs as this one's
+                              thread blocks leave.  By this value the caller states that NONE OF THE CALL'S INPUTS
+                              IS WRITTEN BY THE LIBRARY CALL ISSUED JUST BEFORE IT ON THE SAME STREAM (they may be
+                              read while that call still runs); outputs and workspace are ordered as always.  Calls
+                              on one workspace alternate between two halves of the quantizer's scratch (the
+                              workspace sizes include both).  Any other library call that follows on the stream is
+                              launched as an ordinary kernel and waits for everything before it.  The paper has no
+                              counterpart: this is a launch configuration for back-to-back latency. */
 } hbl_path_t;
 
 const char* hbl_status_string(int status);

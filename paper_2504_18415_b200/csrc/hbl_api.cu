@@ -2,6 +2,8 @@
 // workspace carving and kernel dispatch.  No device memory is allocated here.
 #include <math.h>
 
+#include <mutex>
+
 #include "hbl_common.cuh"
 
 using namespace hbl;
@@ -35,6 +37,51 @@ int sm_count() {
   return cached[dev];
 }
 
+// ---- host-side memory of early-releasing launches (see launch_dependent) ----
+namespace {
+std::mutex g_overlap_mutex;
+constexpr int kStreamSlots = 64, kWorkspaceSlots = 256;
+struct StreamSlot { cudaStream_t s; bool used, early; } g_streams[kStreamSlots] = {};
+bool g_stream_overflow = false;       // an early release on a stream that found no slot: every unknown stream counts as early
+struct WorkspaceSlot { const void* ws; bool used; int last; } g_workspaces[kWorkspaceSlots] = {};
+}
+LaunchMode& launch_mode() {
+  static thread_local LaunchMode mode;
+  return mode;
+}
+bool stream_released_early(cudaStream_t s) {
+  std::lock_guard<std::mutex> lock(g_overlap_mutex);
+  for (int i = 0; i < kStreamSlots; ++i)
+    if (g_streams[i].used && g_streams[i].s == s) return g_streams[i].early;
+  return g_stream_overflow;
+}
+void set_stream_released_early(cudaStream_t s, bool v) {
+  std::lock_guard<std::mutex> lock(g_overlap_mutex);
+  int free_slot = -1;
+  for (int i = 0; i < kStreamSlots; ++i) {
+    if (g_streams[i].used && g_streams[i].s == s) { g_streams[i].early = v; return; }
+    if (!g_streams[i].used && free_slot < 0) free_slot = i;
+  }
+  if (!v && !g_stream_overflow) return;                       // nothing to remember
+  if (free_slot >= 0) g_streams[free_slot] = {s, true, v};
+  else if (v) g_stream_overflow = true;
+}
+namespace {
+// Which half of the double-buffered activation scratch the next overlapping call on this workspace writes:
+// the one the call before it did not (0, 1, 0, ...); -1 when the table is full (the call then runs unoverlapped).
+int next_overlap_half(const void* ws) {
+  std::lock_guard<std::mutex> lock(g_overlap_mutex);
+  int free_slot = -1;
+  for (int i = 0; i < kWorkspaceSlots; ++i) {
+    if (g_workspaces[i].used && g_workspaces[i].ws == ws) { g_workspaces[i].last ^= 1; return g_workspaces[i].last; }
+    if (!g_workspaces[i].used && free_slot < 0) free_slot = i;
+  }
+  if (free_slot < 0) return -1;
+  g_workspaces[free_slot] = {ws, true, 0};
+  return 0;
+}
+}  // namespace
+
 namespace {
 unsigned long long g_launches = 0;
 // One slot per kernel class, so that several classes can be bracketed during the same calls.
@@ -65,6 +112,7 @@ constexpr int kMaxInDim = 32768;
 struct ForwardWs {           // byte offsets inside the caller's workspace
   size_t scale, codesum, zero_region, counters, acc, codes, w_i8, total;
   size_t zero_words;
+  size_t second_half;        // where the second copy of [scale, w_i8) starts (calls in HBL_PATH_STREAM_OVERLAP alternate); 0: none
 };
 
 ForwardWs carve(int T, int K, int N) {
@@ -80,9 +128,18 @@ ForwardWs carve(int T, int K, int N) {
   off = align_up(off, 1024);
   w.codes = off;   off = align_up(off + (size_t)T * K, 1024);
   w.w_i8 = off;    off = align_up(off + (size_t)N * K, 1024);
+  if (T <= kStreamMaxTokens) { w.second_half = off; off += w.w_i8; }
   w.total = off;
   return w;
 }
+
+// Sets what launch_dependent() reads for the launches of one call, and clears it when the call returns.
+struct OverlapScope {
+  explicit OverlapScope(bool on) { launch_mode().overlap_ok = on; }
+  ~OverlapScope() { launch_mode().overlap_ok = false; launch_mode().releases_early = false; }
+};
+// SMs a contraction that releases early leaves to the next call's quantizer: its thread blocks come two to an SM.
+int overlap_reserve(long act_threads) { return (int)((act_threads + 511) / 512); }
 
 int check_dims(int tokens, int in_dim, int out_dim) {
   if (tokens < 0 || in_dim <= 0 || out_dim <= 0) return HBL_ERR_SHAPE;
@@ -111,7 +168,7 @@ int resolve_path(int path, int tokens, size_t packed_bytes, int n_tensors) {
     if (tokens <= limit && packed_bytes >= (size_t)16 << 20) return HBL_PATH_STREAM;
     return HBL_PATH_TENSOR;
   }
-  if (path == HBL_PATH_STREAM) return tokens <= kStreamMaxTokens ? HBL_PATH_STREAM : -1;
+  if (path == HBL_PATH_STREAM || path == HBL_PATH_STREAM_OVERLAP) return tokens <= kStreamMaxTokens ? path : -1;
   if (path == HBL_PATH_TENSOR || path == HBL_PATH_TENSOR_PACKED) return path;
   return -2;
 }
@@ -278,13 +335,18 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   const ForwardWs w = carve(tokens, in_dim, out_dim);
   if (workspace_bytes < w.total) return HBL_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  char* ws = static_cast<char*>(workspace);
+  // back-to-back mode: this call's quantizer may run beside the previous call's contraction, so it writes the half
+  // of the scratch that call does not read (no slot left to remember the workspace: an ordinary streaming call)
+  const int half = (p == HBL_PATH_STREAM_OVERLAP) ? next_overlap_half(workspace) : -1;
+  const bool overlap = half >= 0;
+  OverlapScope scope(overlap);
+  char* ws = static_cast<char*>(workspace) + (half == 1 ? w.second_half : 0);
   float* scale = reinterpret_cast<float*>(ws + w.scale);
   int32_t* codesum = reinterpret_cast<int32_t*>(ws + w.codesum);
   int8_t* codes = reinterpret_cast<int8_t*>(ws + w.codes);
-  const bool stream_path = (p == HBL_PATH_STREAM);
+  const bool stream_path = (p == HBL_PATH_STREAM || p == HBL_PATH_STREAM_OVERLAP);
   SidePipe* sp = nullptr;
-  int8_t* w_i8 = reinterpret_cast<int8_t*>(ws + w.w_i8);
+  int8_t* w_i8 = reinterpret_cast<int8_t*>(static_cast<char*>(workspace) + w.w_i8);
   if (!stream_path) {
     // the weights are expanded on the side stream while the activations are quantized on the caller's
     sp = side_pipe();
@@ -308,7 +370,8 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   if (stream_path)
     return launch_gemm_stream(codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha,
                               static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
-                              reinterpret_cast<int*>(ws + w.counters), s);
+                              reinterpret_cast<int*>(ws + w.counters), s,
+                              overlap ? overlap_reserve((long)tokens * (in_dim / 64 < 32 ? 32 : in_dim / 64)) : -1);
   HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[0], 0));
   return launch_gemm_tensor(codes, packed, scale, tokens, in_dim, w_i8, out_dim, alpha, static_cast<__nv_bfloat16*>(y), nullptr, s);
 }
@@ -390,6 +453,7 @@ int hbl_norm_quantize_act(const void* x, const void* gain, int gain_dtype, float
 namespace {
 struct BlockWs {
   size_t scale[4], codesum[4], codes[4], zero_region, counters[7], acc[7], w_i8, total, zero_words;
+  size_t second_half;        // as in ForwardWs
 };
 BlockWs carve_block(int T, int H, int F) {
   BlockWs w{};
@@ -406,6 +470,7 @@ BlockWs carve_block(int T, int H, int F) {
   off = align_up(off, 1024);
   for (int i = 0; i < 4; ++i) { w.codes[i] = off; off = align_up(off + (size_t)T * in_dims[i], 1024); }
   w.w_i8 = off; off = align_up(off + 3 * align_up((size_t)F * H, 1024), 1024);   // three buffers of the largest weight (F x H)
+  if (T <= kStreamMaxTokens) { w.second_half = off; off += w.w_i8; }
   w.total = off;
   return w;
 }
@@ -451,10 +516,15 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   const BlockWs w = carve_block(T, H, F);
   if (workspace_bytes < w.total) return HBL_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  char* ws = static_cast<char*>(workspace);
+  // back-to-back mode (not for the chained feed-forward block, whose second quantizer reads the first launch's
+  // outputs): see forward_impl
+  const int half = (p == HBL_PATH_STREAM_OVERLAP && !chain_ffn) ? next_overlap_half(workspace) : -1;
+  const bool overlap = half >= 0;
+  OverlapScope scope(overlap);
+  char* ws = static_cast<char*>(workspace) + (half == 1 ? w.second_half : 0);
   const int in_dims[4] = {H, H, H, F};
   const int had[4] = {0, 1, 0, 1};
-  const bool stream_path = (p == HBL_PATH_STREAM);
+  const bool stream_path = (p == HBL_PATH_STREAM || p == HBL_PATH_STREAM_OVERLAP);
   SidePipe* sp = nullptr;
   if (!stream_path) {
     // fork the side stream now: its first expansions overlap the quantizations below, and it starts
@@ -505,7 +575,11 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
       jobs[i] = {Ws[i], b->alpha7 + i, static_cast<__nv_bfloat16*>(ys[i]), nullptr, out_dims[i], src[i]};
     int32_t* part = reinterpret_cast<int32_t*>(ws + w.acc[0]);
     int* flags = reinterpret_cast<int*>(ws + w.counters[0]);
-    if (!chain_ffn) return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, part, flags, s);
+    if (!chain_ffn) {
+      long act_threads = 0;                                   // of the next call's quantizer, which has this call's shape
+      for (int i = 0; i < 4; ++i) act_threads += (long)T * (in_dims[i] / 64);
+      return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, part, flags, s, overlap ? overlap_reserve(act_threads) : -1);
+    }
     // chained: six projections, then the gating product + quantizer (which also clears the flags again: it
     // starts only when the first launch has completed), then the down projection
     rc = launch_gemm_stream_multi(inputs, 3, jobs, 6, T, part, flags, s);
@@ -783,7 +857,7 @@ int hbl_gemm_i32(const int8_t* codes, const int32_t* codesum, int tokens, int in
   if (rc != HBL_OK) return rc;
   const int p = resolve_path(path, tokens, (size_t)out_dim * in_dim / 4, 1);
   if (p == -1) return HBL_ERR_TOO_LARGE;
-  if (p < 0) return HBL_ERR_FORMAT;
+  if (p < 0 || p == HBL_PATH_STREAM_OVERLAP) return HBL_ERR_FORMAT;   // (the caller's codes: nothing here to run beside a previous call)
   if (tokens == 0) return HBL_OK;
   if (!codes || !W_packed || !acc_out || !workspace) return HBL_ERR_NULL;
   if (p == HBL_PATH_TENSOR_PACKED) return HBL_ERR_FORMAT;      // these codes are one per byte: see hbl_gemm_i32_int4_packed

@@ -61,9 +61,26 @@ int sm_count();   // multiprocessors of the current device (148 if the query fai
 // The dependent must call grid_dependency_wait() before it reads anything the earlier kernel
 // writes.  The activation kernels also call it last thing, so that "kernel k has completed"
 // implies "kernels before k have completed" along a chain of such launches.
+//
+// One kernel releases its dependents long before it ends: the streaming contraction of a call made with
+// HBL_PATH_STREAM_OVERLAP.  What follows it may then run beside it, which only a call in the same mode is
+// prepared for (it writes to the other half of a double-buffered workspace, and its caller has stated that its
+// inputs do not come from the call before).  The library therefore remembers, per stream, whether its last
+// launch was such a kernel, and gives the next launch on that stream the programmatic attribute only if that
+// launch belongs to a call in the same mode; any other launch is an ordinary one and starts when everything
+// before it is complete.  LaunchMode is what the entry point in charge sets for the launches it makes.
+struct LaunchMode {
+  bool overlap_ok = false;            // the launches of this call may run beside an early-releasing contraction
+  bool releases_early = false;        // the next launch is such a contraction
+};
+LaunchMode& launch_mode();                                    // per host thread
+bool stream_released_early(cudaStream_t s);                   // the library's last launch on s releases early
+void set_stream_released_early(cudaStream_t s, bool v);
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
                                     Args... args) {
+  const LaunchMode mode = launch_mode();
+  const bool programmatic = mode.overlap_ok || !stream_released_early(s);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -71,10 +88,12 @@ inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 bloc
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[0].val.programmaticStreamSerializationAllowed = programmatic ? 1 : 0;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+  set_stream_released_early(s, mode.releases_early);
+  return e;
 }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -122,9 +141,12 @@ struct GemmSegment {          // one weight tensor of a (possibly fused) project
   void* y;                    // bf16 [T, N]
   int N;
 };
+// early_release_reserve >= 0 (calls in HBL_PATH_STREAM_OVERLAP): the kernel releases its programmatic dependents as
+// soon as it has seen the kernel before it complete, and leaves that many SMs without a thread block of its own
+// for the next call's quantizer to run on; -1: neither.
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
                        const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
-                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s);
+                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s, int early_release_reserve = -1);
 // Several weight tensors that read the same quantized input (q | k | v, up | gate), contracted as ONE matrix of
 // concatenated weight rows: output i takes the rows [begin[i], begin[i] + width[i]) of W_i8, has its own alpha
 // and its own bf16 tensor [T, width[i]].  begin[0] = 0, the widths of all but the last are multiples of 256.
@@ -145,7 +167,7 @@ int gemm_stream_max_tokens();
 struct StreamInput { const int8_t* codes; const float* scale; const int32_t* codesum; int K; };
 struct StreamJob { const void* W_packed; const float* alpha; __nv_bfloat16* y; int32_t* acc_out; int N; int input; };
 int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
-                             int32_t* part, int* flags, cudaStream_t s);
+                             int32_t* part, int* flags, cudaStream_t s, int early_release_reserve = -1);
 size_t gemm_stream_acc_words(int T, int N);       // int32 words of split-K scratch (0 if none)
 size_t gemm_stream_counter_words(int N);
 

@@ -14,7 +14,7 @@ import torch
 
 HBL_OK = 0
 HBL_F32, HBL_BF16 = 0, 1
-PATH_AUTO, PATH_STREAM, PATH_TENSOR, PATH_TENSOR_PACKED = 0, 1, 2, 3
+PATH_AUTO, PATH_STREAM, PATH_TENSOR, PATH_TENSOR_PACKED, PATH_STREAM_OVERLAP = 0, 1, 2, 3, 4
 
 STATUS_NAMES = {
     0: "HBL_OK", 1: "HBL_ERR_NULL", 2: "HBL_ERR_SHAPE", 3: "HBL_ERR_NOT_POW2", 4: "HBL_ERR_BITS",

@@ -55,6 +55,7 @@ def test_argument_errors_come_before_any_launch(L):
     assert f(dt=7) == 10                       # HBL_ERR_FORMAT
     assert f(path=9) == 10
     assert f(T=600, path=hbl.PATH_STREAM) == 11   # HBL_ERR_TOO_LARGE
+    assert f(T=600, path=hbl.PATH_STREAM_OVERLAP) == 11
     assert f(K=65536) == 11
     assert f(T=0) == 0                         # no-op
     assert f(x=n) == 1                         # HBL_ERR_NULL
@@ -85,6 +86,7 @@ def test_argument_errors_come_before_any_launch(L):
     assert L.hbl_hadamard_bf16(p, 0, 4096, p, n) == 0            # no tokens: no-op
     assert L.hbl_quantize_act(p, 0, 4, 512, 3, 1, 1e-5, p, p, p, n) == 4
     assert L.hbl_gemm_i32(p, n, 4, 512, p, 512, p, p, 1 << 30, hbl.PATH_STREAM, n) == 1   # codesum required
+    assert L.hbl_gemm_i32(p, p, 4, 512, p, 512, p, p, 1 << 30, hbl.PATH_STREAM_OVERLAP, n) == 10   # quantizing calls only
     kv = lambda **kw: L.hbl_quantize_kv(kw.get("x", p), kw.get("T", 4), kw.get("H", 8), kw.get("D", 128), kw.get("bits", 4),
                                         kw.get("S", 0), kw.get("eps", 1e-5), kw.get("codes", p), kw.get("scale", p),
                                         kw.get("bos", n), kw.get("bos_scale", n), n)
