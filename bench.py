@@ -203,6 +203,19 @@ def time_loop(fn, iters, warmup, torch):
     return e0.elapsed_time(e1) / iters
 
 
+def graph_ms(call, ring, reps, torch):
+    """ms per call of `ring` back-to-back calls captured in one CUDA graph (launch latencies hide one another)."""
+    for _ in range(2):
+        for _ in range(ring):
+            call()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(ring):
+            call()
+    return time_loop(g.replay, reps, 3, torch) / ring
+
+
 def layer_point(name, kind, seed, K, N, bits, had, T, torch, hbl, peaks, iters=None):
     """One single-layer workload point, L2-cold (ring of distinct input sets), returns a dict."""
     per_call = alg_bytes(T, K, N) + T * K          # + the int8 codes round trip (implementation traffic)
@@ -217,28 +230,23 @@ def layer_point(name, kind, seed, K, N, bits, had, T, torch, hbl, peaks, iters=N
         ys.append(torch.empty((T, N), dtype=torch.bfloat16, device="cuda"))
     wsb = hbl.hbl_workspace_bytes(T, K, N)
     work = hbl.new_workspace(wsb)
-    path = hbl.PATH_AUTO
-    state = {"i": 0}
+    state = {"i": 0, "path": hbl.PATH_AUTO}
 
     def call():
         r = state["i"] % ring
         state["i"] += 1
-        hbl.hbl_forward(xs[r], ws[r][0], ws[r][1], N, bits, had, EPS, y=ys[r], workspace=work, path=path)
+        hbl.hbl_forward(xs[r], ws[r][0], ws[r][1], N, bits, had, EPS, y=ys[r], workspace=work, path=state["path"])
 
     small = T <= 512                     # the streaming path: a few launches per call, timed as a CUDA graph
+    ms_b2b = None
     if small:
-        # launch-latency hiding: one CUDA graph of `ring` back-to-back calls
-        for _ in range(2):
-            for _ in range(ring):
-                call()
-        torch.cuda.synchronize()
-        state["i"] = 0
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            for _ in range(ring):
-                call()
-        reps = iters or 20
-        ms = time_loop(g.replay, reps, 3, torch) / ring
+        ms = graph_ms(call, ring, iters or 20, torch)
+        # the same calls in the library's back-to-back mode (no input here is written by the call before it), where
+        # the automatic choice is the streaming kernel that mode is built on (the library's rule: up to 128 tokens,
+        # or up to 192 with 16 MiB or more of packed weights)
+        if T <= 128 or (T <= 192 and N * K // 4 >= 16 << 20):
+            state["i"], state["path"] = 0, hbl.PATH_STREAM_OVERLAP
+            ms_b2b = graph_ms(call, ring, iters or 20, torch)
     else:
         flops = 2.0 * T * K * N
         est_ms = max(0.02, flops / 2.0e15 * 1e3)
@@ -256,6 +264,9 @@ def layer_point(name, kind, seed, K, N, bits, had, T, torch, hbl, peaks, iters=N
         out["bound"] = "hbm"
         out["frac"] = round(gbs / peaks["hbm_gbs"], 4)
         out["frac_of_nominal_hbm"] = round(gbs / NOMINAL_HBM_GBS, 4)
+        if ms_b2b is not None:
+            out["ms_back_to_back_mode"] = round(ms_b2b, 5)
+            out["frac_back_to_back_mode"] = round(alg_bytes(T, K, N) / (ms_b2b * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)
     else:
         out["bound"] = "tensor"
         out["frac"] = round(tops / (2 * peaks["bf16_tflops"]), 4)
@@ -483,23 +494,18 @@ def block_point(T, torch, hbl, peaks, iters=None):
     dims = {"q": H, "k": H, "v": H, "o": H, "up": F, "gate": F, "down": H}
     outs = {n: torch.empty((T, d), dtype=torch.bfloat16, device="cuda") for n, d in dims.items()}
     work = hbl.new_workspace(hbl.hbl_block_workspace_bytes(T, H, F))
-    state = {"i": 0}
+    state = {"i": 0, "path": hbl.PATH_AUTO}
 
     def call():
         r = state["i"] % ring
         state["i"] += 1
-        hbl.hbl_block_forward(ins, sets[r][0], sets[r][1], H, F, 4, EPS, outputs=outs, workspace=work)
+        hbl.hbl_block_forward(ins, sets[r][0], sets[r][1], H, F, 4, EPS, outputs=outs, workspace=work, path=state["path"])
 
+    ms_b2b = None
     if small:
-        for _ in range(2 * ring):
-            call()
-        torch.cuda.synchronize()
-        state["i"] = 0
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            for _ in range(ring):
-                call()
-        ms = time_loop(g.replay, iters or 10, 3, torch) / ring
+        ms = graph_ms(call, ring, iters or 10, torch)
+        state["i"], state["path"] = 0, hbl.PATH_STREAM_OVERLAP
+        ms_b2b = graph_ms(call, ring, iters or 10, torch)
     else:
         flops = 2.0 * T * sum(n * k for n, k in shapes.values())
         est_ms = flops / 2.0e15 * 1e3
@@ -515,6 +521,9 @@ def block_point(T, torch, hbl, peaks, iters=None):
     if tops < 100 or small:
         out["bound"] = "hbm"; out["frac"] = round(gbs / peaks["hbm_gbs"], 4)
         out["frac_of_nominal_hbm"] = round(gbs / NOMINAL_HBM_GBS, 4)
+        if ms_b2b is not None:
+            out["ms_back_to_back_mode"] = round(ms_b2b, 5)
+            out["frac_back_to_back_mode"] = round(per_call / (ms_b2b * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)
     else:
         out["bound"] = "tensor"; out["frac"] = round(tops / (2 * peaks["bf16_tflops"]), 4)
         out["frac_of_sustained"] = round(tops / (2 * peaks["bf16_tflops_sustained"]), 4)
