@@ -243,8 +243,8 @@ def layer_point(name, kind, seed, K, N, bits, had, T, torch, hbl, peaks, iters=N
         ms = graph_ms(call, ring, iters or 20, torch)
         # the same calls in the library's back-to-back mode (no input here is written by the call before it), where
         # the automatic choice is the streaming kernel that mode is built on (the library's rule: up to 128 tokens,
-        # or up to 192 with 16 MiB or more of packed weights)
-        if T <= 128 or (T <= 192 and N * K // 4 >= 16 << 20):
+        # up to 192 with 16 MiB or more of packed weights, up to 256 with 32 MiB or more)
+        if T <= 128 or (T <= 192 and N * K // 4 >= 16 << 20) or (T <= 256 and N * K // 4 >= 32 << 20):
             state["i"], state["path"] = 0, hbl.PATH_STREAM_OVERLAP
             ms_b2b = graph_ms(call, ring, iters or 20, torch)
     else:

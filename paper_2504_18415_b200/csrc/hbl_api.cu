@@ -159,12 +159,12 @@ int check_quant_args(int x_dtype, int in_dim, int bits, int use_hadamard, float 
 // Which contraction kernel.  The streaming kernel reads the packed weights once per 128 tokens; the
 // large-batch path pays an expansion and a launch per weight tensor.  Measured cross-overs: one pass
 // (<= 128 tokens) always goes to the streaming kernel; a single layer of 16 MiB or more of packed weights
-// up to 192 tokens (at 256 the two are level, beyond it the large-batch path wins: 32 MiB at 512 tokens
-// 161 vs 104 us); the seven tensors of a decoder block up to 512 tokens (64 MiB: 271 vs 268 us there).
+// up to 192 tokens, of 32 MiB or more up to 256 (32 MiB: 63 vs 81 us at 256 tokens, 95 vs 92 at 384,
+// 126 vs 105 at 512); the seven tensors of a decoder block up to 512 tokens (64 MiB: 237 vs 246 us there).
 int resolve_path(int path, int tokens, size_t packed_bytes, int n_tensors) {
   if (path == HBL_PATH_AUTO) {
     if (tokens <= 128) return HBL_PATH_STREAM;
-    const int limit = n_tensors > 1 ? kStreamMaxTokens : 192;
+    const int limit = n_tensors > 1 ? kStreamMaxTokens : (packed_bytes >= ((size_t)32 << 20) ? 256 : 192);
     if (tokens <= limit && packed_bytes >= (size_t)16 << 20) return HBL_PATH_STREAM;
     return HBL_PATH_TENSOR;
   }
