@@ -69,7 +69,9 @@ typedef enum {
                               IS WRITTEN BY THE LIBRARY CALL ISSUED JUST BEFORE IT ON THE SAME STREAM (they may be
                               read while that call still runs); outputs and workspace are ordered as always.  Calls
                               on one workspace alternate between two halves of the quantizer's scratch (the
-                              workspace sizes include both).  Any other library call that follows on the stream is
+                              workspace sizes include both); with bf16 inputs the contraction starts on an input's
+                              codes as soon as all thread blocks of the quantizer have counted themselves in for it
+                              (counters in device memory of the library, 256 workspaces remembered per process).  Any other library call that follows on the stream is
                               launched as an ordinary kernel and waits for everything before it.  The paper has no
                               counterpart: this is a launch configuration for back-to-back latency. */
 } hbl_path_t;
@@ -213,7 +215,10 @@ unsigned long long hbl_launch_count(void);
 int hbl_profile_events(void** start_events, void** stop_events, int n, int kernel);
 
 /* Synchronises `stream`, returns the first device-side error recorded since the
- * last call (HBL_OK if none) and clears it. */
+ * last call (HBL_OK if none) and clears it.  After an error it also clears the
+ * counters HBL_PATH_STREAM_OVERLAP keeps in device memory of the library (the
+ * quantizer's thread blocks count themselves in there; a kernel that gave up may
+ * have left them mid-count). */
 int hbl_check_status(void* stream);
 
 /* Test aid (no counterpart in the paper): makes a bounded device-side wait run out on purpose.  One small

@@ -652,7 +652,15 @@ struct ActMultiParams {
   float eps;
   int32_t* zero_fill;
   size_t zero_words;
+  unsigned* ready;                    // per input: thread blocks that have written their codes (nullptr: not counted)
 };
+
+// Last thing a thread block does: its stores are made visible, then one thread counts the block in.
+__device__ __forceinline__ void count_block_in(unsigned* counter) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) atomicAdd(counter, 1u);
+}
 
 template <int BITS>
 __global__ void __launch_bounds__(kMultiThreads)
@@ -671,6 +679,7 @@ act_multi_bf16_kernel(const __grid_constant__ ActMultiParams p) {
   const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(job.x);
   if (!job.use_hadamard) {
     quant_rows_bf16_body<BITS>(x, p.T, job.K, p.nt[j], p.eps, job.codes, job.scale, job.codesum, 0, block, red_f, red_i);
+    if (p.ready != nullptr) count_block_in(p.ready + j);
     grid_dependency_wait();   // chain: this kernel is complete only when the one before it is
     return;
   }
@@ -684,6 +693,7 @@ act_multi_bf16_kernel(const __grid_constant__ ActMultiParams p) {
     default: break;
   }
 #undef HBL_CASE
+  if (p.ready != nullptr) count_block_in(p.ready + j);
   grid_dependency_wait();
 }
 
@@ -699,7 +709,7 @@ bool act_multi_bf16_supported(const ActJob* jobs, int n_jobs) {
 }
 
 int launch_act_multi_bf16(const ActJob* jobs, int n_jobs, int T, int bits, float eps, int32_t* zero_fill,
-                          size_t zero_fill_words, cudaStream_t s) {
+                          size_t zero_fill_words, cudaStream_t s, unsigned* ready, unsigned* blocks_out) {
   if (T <= 0) return HBL_OK;
   if (!act_multi_bf16_supported(jobs, n_jobs)) return HBL_ERR_SHAPE;
   if (bits != 4 && bits != 8) return HBL_ERR_BITS;
@@ -721,6 +731,7 @@ int launch_act_multi_bf16(const ActJob* jobs, int n_jobs, int T, int bits, float
       tpc = kMultiThreads / p.nt[j];
     }
     blocks += (T + tpc - 1) / tpc;
+    if (blocks_out != nullptr) blocks_out[j] = (unsigned)((T + tpc - 1) / tpc);
   }
   p.first_block[n_jobs] = blocks;
   p.n = n_jobs;
@@ -728,6 +739,7 @@ int launch_act_multi_bf16(const ActJob* jobs, int n_jobs, int T, int bits, float
   p.eps = eps;
   p.zero_fill = zero_fill;
   p.zero_words = zero_fill_words;
+  p.ready = ready;
   auto kern = bits == 8 ? act_multi_bf16_kernel<8> : act_multi_bf16_kernel<4>;
   // (the attribute is set once per device, to the most any supported input needs: 2^14 floats)
   if (bits == 8) HBL_ALLOW_DYNAMIC_SMEM(act_multi_bf16_kernel<8>, kMultiMaxSmem);

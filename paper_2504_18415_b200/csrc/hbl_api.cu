@@ -69,16 +69,32 @@ void set_stream_released_early(cudaStream_t s, bool v) {
 namespace {
 // Which half of the double-buffered activation scratch the next overlapping call on this workspace writes:
 // the one the call before it did not (0, 1, 0, ...); -1 when the table is full (the call then runs unoverlapped).
-int next_overlap_half(const void* ws) {
+int next_overlap_half(const void* ws, int* slot) {
   std::lock_guard<std::mutex> lock(g_overlap_mutex);
   int free_slot = -1;
   for (int i = 0; i < kWorkspaceSlots; ++i) {
-    if (g_workspaces[i].used && g_workspaces[i].ws == ws) { g_workspaces[i].last ^= 1; return g_workspaces[i].last; }
+    if (g_workspaces[i].used && g_workspaces[i].ws == ws) { g_workspaces[i].last ^= 1; *slot = i; return g_workspaces[i].last; }
     if (!g_workspaces[i].used && free_slot < 0) free_slot = i;
   }
   if (free_slot < 0) return -1;
   g_workspaces[free_slot] = {ws, true, 0};
+  *slot = free_slot;
   return 0;
+}
+// Counters of the back-to-back mode, per remembered workspace and half: [0..3] thread blocks of the quantizer that
+// have written input m's codes, [4] thread blocks of the contraction that are through.  Zero when the module is
+// loaded; the contraction's last thread block puts them back to zero, so they are zero whenever a call starts.
+__device__ unsigned g_overlap_counters[kWorkspaceSlots][2][8];
+unsigned* overlap_counters(int slot, int half) {
+  static unsigned* base[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return nullptr;
+  if (base[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_overlap_counters) != cudaSuccess) return nullptr;
+    base[dev] = static_cast<unsigned*>(p);
+  }
+  return base[dev] + ((size_t)slot * 2 + half) * 8;
 }
 }  // namespace
 
@@ -337,7 +353,8 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // back-to-back mode: this call's quantizer may run beside the previous call's contraction, so it writes the half
   // of the scratch that call does not read (no slot left to remember the workspace: an ordinary streaming call)
-  const int half = (p == HBL_PATH_STREAM_OVERLAP) ? next_overlap_half(workspace) : -1;
+  int slot = -1;
+  const int half = (p == HBL_PATH_STREAM_OVERLAP) ? next_overlap_half(workspace, &slot) : -1;
   const bool overlap = half >= 0;
   OverlapScope scope(overlap);
   char* ws = static_cast<char*>(workspace) + (half == 1 ? w.second_half : 0);
@@ -360,6 +377,21 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   int32_t* zf = stream_path ? reinterpret_cast<int32_t*>(ws + w.zero_region) : nullptr;
   const size_t zw = stream_path ? w.zero_words : 0;
   int32_t* cs = stream_path ? codesum : nullptr;             // only the streaming kernel needs the code sums
+  if (overlap && !gain && !up && x_dtype == HBL_BF16) {
+    // the quantizer whose thread blocks count themselves in, so that the contraction can start on the codes while
+    // the call before this one is still draining
+    const ActJob job = {x, codes, scale, codesum, in_dim, use_hadamard};
+    unsigned* counters = overlap_counters(slot, half);
+    if (counters != nullptr && act_multi_bf16_supported(&job, 1)) {
+      StreamReady ready = {counters, {0, 0, 0, 0}, counters + 4};
+      rc = launch_act_multi_bf16(&job, 1, tokens, bits, eps, zf, zw, s, counters, ready.target);
+      if (rc != HBL_OK) return rc;
+      return launch_gemm_stream(codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha,
+                                static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
+                                reinterpret_cast<int*>(ws + w.counters), s,
+                                overlap_reserve((long)tokens * (in_dim / 64 < 32 ? 32 : in_dim / 64)), &ready);
+    }
+  }
   rc = gain ? launch_norm_act_quant_bf16(x, gain, gain_dtype, norm_eps, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s, packed)
        : up ? launch_glu_act_quant_bf16(x, up, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s, packed)
             : launch_act_quant(x, x_dtype, tokens, in_dim, bits, use_hadamard, eps, codes, scale, cs, nullptr, zf, zw, s, packed);
@@ -518,7 +550,8 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // back-to-back mode (not for the chained feed-forward block, whose second quantizer reads the first launch's
   // outputs): see forward_impl
-  const int half = (p == HBL_PATH_STREAM_OVERLAP && !chain_ffn) ? next_overlap_half(workspace) : -1;
+  int slot = -1;
+  const int half = (p == HBL_PATH_STREAM_OVERLAP && !chain_ffn) ? next_overlap_half(workspace, &slot) : -1;
   const bool overlap = half >= 0;
   OverlapScope scope(overlap);
   char* ws = static_cast<char*>(workspace) + (half == 1 ? w.second_half : 0);
@@ -542,14 +575,17 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   // or two, which is what a call of a few tokens spends most of its time on besides the weights)
   const int n_act = chain_ffn ? 3 : 4;
   bool one_launch = false;
+  StreamReady ready = {nullptr, {0, 0, 0, 0}, nullptr};     // back-to-back mode: the quantizer's thread blocks count themselves in
   if (stream_path && b->x_dtype == HBL_BF16) {
     ActJob aj[4];
     for (int i = 0; i < n_act; ++i)
       aj[i] = {xs[i], reinterpret_cast<int8_t*>(ws + w.codes[i]), reinterpret_cast<float*>(ws + w.scale[i]),
                reinterpret_cast<int32_t*>(ws + w.codesum[i]), in_dims[i], had[i]};
     if (act_multi_bf16_supported(aj, n_act)) {
+      unsigned* counters = overlap ? overlap_counters(slot, half) : nullptr;
+      if (counters != nullptr) ready = {counters, {0, 0, 0, 0}, counters + 4};
       rc = launch_act_multi_bf16(aj, n_act, T, b->bits, b->eps, reinterpret_cast<int32_t*>(ws + w.zero_region),
-                                 w.zero_words, s);
+                                 w.zero_words, s, counters, ready.target);
       if (rc != HBL_OK) return rc;
       one_launch = true;
     }
@@ -578,7 +614,8 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     if (!chain_ffn) {
       long act_threads = 0;                                   // of the next call's quantizer, which has this call's shape
       for (int i = 0; i < 4; ++i) act_threads += (long)T * (in_dims[i] / 64);
-      return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, part, flags, s, overlap ? overlap_reserve(act_threads) : -1);
+      return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, part, flags, s, overlap ? overlap_reserve(act_threads) : -1,
+                                      ready.ready != nullptr ? &ready : nullptr);
     }
     // chained: six projections, then the gating product + quantizer (which also clears the flags again: it
     // starts only when the first launch has completed), then the down projection
@@ -780,6 +817,12 @@ int hbl_check_status(void* stream) {
   int st = 0;
   if (cudaMemcpy(&st, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return HBL_ERR_CUDA;
   if (st != 0 && cudaMemset(word, 0, sizeof(int)) != cudaSuccess) return HBL_ERR_CUDA;
+  if (st != 0) {
+    // a kernel that gave up may have left the back-to-back mode's counters mid-count: back to zero (the stream was
+    // synchronised above; calls on other streams of this device must not be in flight, as for the status word)
+    unsigned* counters = overlap_counters(0, 0);
+    if (counters == nullptr || cudaMemset(counters, 0, sizeof(unsigned) * kWorkspaceSlots * 2 * 8) != cudaSuccess) return HBL_ERR_CUDA;
+  }
   return st;
 }
 

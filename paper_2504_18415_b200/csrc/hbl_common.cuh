@@ -112,8 +112,10 @@ bool act_quant_bf16_supported(int K);
 constexpr int kMaxActJobs = 4;
 struct ActJob { const void* x; int8_t* codes; float* scale; int32_t* codesum; int K; int use_hadamard; };
 bool act_multi_bf16_supported(const ActJob* jobs, int n_jobs);
+// ready (optional): n_jobs counters; every thread block adds one to its input's when its codes, scales and code
+// sums are written.  blocks_out (optional): thread blocks per input.
 int launch_act_multi_bf16(const ActJob* jobs, int n_jobs, int T, int bits, float eps, int32_t* zero_fill,
-                          size_t zero_fill_words, cudaStream_t s);
+                          size_t zero_fill_words, cudaStream_t s, unsigned* ready = nullptr, unsigned* blocks_out = nullptr);
 int launch_act_quant_bf16(const void* x, int T, int K, int bits, float eps, int8_t* codes, float* scale,
                           int32_t* codesum, float* xr_out, int32_t* zero_fill, size_t zero_fill_words,
                           cudaStream_t s, bool packed = false);
@@ -144,9 +146,14 @@ struct GemmSegment {          // one weight tensor of a (possibly fused) project
 // early_release_reserve >= 0 (calls in HBL_PATH_STREAM_OVERLAP): the kernel releases its programmatic dependents as
 // soon as it has seen the kernel before it complete, and leaves that many SMs without a thread block of its own
 // for the next call's quantizer to run on; -1: neither.
+// ready (same mode, optional): counters the quantizer's thread blocks raise per input when their codes are written
+// (target[m] thread blocks for input m); the contraction then starts on an input's codes as soon as they are all
+// there instead of when the quantizer has completed, and its last thread block clears the counters and `done`.
+struct StreamReady { unsigned* ready; unsigned target[4]; unsigned* done; };
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
                        const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
-                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s, int early_release_reserve = -1);
+                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s, int early_release_reserve = -1,
+                       const StreamReady* ready = nullptr);
 // Several weight tensors that read the same quantized input (q | k | v, up | gate), contracted as ONE matrix of
 // concatenated weight rows: output i takes the rows [begin[i], begin[i] + width[i]) of W_i8, has its own alpha
 // and its own bf16 tensor [T, width[i]].  begin[0] = 0, the widths of all but the last are multiples of 256.
@@ -167,7 +174,8 @@ int gemm_stream_max_tokens();
 struct StreamInput { const int8_t* codes; const float* scale; const int32_t* codesum; int K; };
 struct StreamJob { const void* W_packed; const float* alpha; __nv_bfloat16* y; int32_t* acc_out; int N; int input; };
 int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
-                             int32_t* part, int* flags, cudaStream_t s, int early_release_reserve = -1);
+                             int32_t* part, int* flags, cudaStream_t s, int early_release_reserve = -1,
+                             const StreamReady* ready = nullptr);
 size_t gemm_stream_acc_words(int T, int N);       // int32 words of split-K scratch (0 if none)
 size_t gemm_stream_counter_words(int N);
 

@@ -71,6 +71,13 @@ struct Params {
   int* status;
   int T;
   int release_early;  // release the programmatic dependents once the kernel before this one is known to be complete
+  // Back-to-back mode: the quantizer of this call ran beside the previous contraction and completes only when that
+  // one does.  Its thread blocks count themselves in per input (ready[m], counters the library owns) once their
+  // codes are written, and the codes producer waits for those counts instead of the quantizer's completion, so the
+  // MMAs start while the previous contraction still drains; the epilogue keeps waiting for completion.
+  const unsigned* ready;          // nullptr: wait for the kernel before this one as a whole
+  unsigned ready_target[MAX_MAPS];
+  unsigned* done;                 // non-null: thread blocks of this launch that are through; the last one clears ready[] and done
 };
 struct CodeMaps { CUtensorMap m[MAX_MAPS]; };   // codes [T, K] of each input, box 128 x T_pad, 128-byte swizzle
 
@@ -102,6 +109,25 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
+}
+// Waits (bounded) until a counter that another kernel's thread blocks raise has reached `target`.  That kernel was
+// launched before this one and waits for nothing this one does.
+__device__ __forceinline__ bool wait_count(const unsigned* counter, unsigned target, volatile int* abort_flag, int* status) {
+  const uint64_t t0 = global_ns();
+  for (uint32_t polls = 0;; ++polls) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) break;
+    if (*abort_flag) return false;
+    if ((polls & 63u) == 63u && global_ns() - t0 > kWaitLimitNs) {
+      report_device_error(status, HBL_ERR_TIMEOUT);
+      *abort_flag = 1;
+      return false;
+    }
+    __nanosleep(100);
+  }
+  asm volatile("fence.proxy.async.global;" ::: "memory");   // the bulk tensor copies that follow read what the counter covers
+  return true;
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -277,16 +303,22 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
   } else if (warp == 2) {
     // ------------------------------ codes producer ------------------------------
     if (lane == 0) {
-      grid_dependency_wait();                                  // the codes come from the previous kernel
-      // (only now: whatever is released runs beside this kernel and may be followed by another contraction; the
-      //  wait above has seen the kernel before this one complete, so at most two calls are ever in flight)
-      if (p.release_early) grid_launch_dependents();
+      uint32_t complete = 0;                                   // inputs whose codes are known to be written
+      if (p.ready == nullptr) {
+        grid_dependency_wait();                                // the codes come from the previous kernel
+        complete = ~0u;
+      }
       Range range(p, u0, u1);
       Segment sg;
       uint32_t i = 0;
       bool ok = true;
       while (ok && range.next(sg)) {
-        const CUtensorMap* tm_codes = &maps.m[p.jobs[sg.job].map];
+        const int in = p.jobs[sg.job].map;
+        if (!((complete >> in) & 1u)) {
+          if (!wait_count(p.ready + in, p.ready_target[in], abort_flag, p.status)) break;
+          complete |= 1u << in;
+        }
+        const CUtensorMap* tm_codes = &maps.m[in];
         for (int kb = sg.ka; kb < sg.ke; ++kb, ++i) {
           const int s = i % SC;
           if (i >= (uint32_t)SC && !mbar_wait<true>(&c_empty[s], ((i / SC) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
@@ -399,6 +431,10 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     // Accumulators are handled 16 token columns at a time, so nothing here needs more than a few
     // dozen registers whatever T_PAD is.
     grid_dependency_wait();                                  // scales, code sums and cleared flags come from the previous kernel
+    // Back-to-back mode: only now may the next call's quantizer start (it runs beside this kernel and may be followed
+    // by another contraction; the wait above has seen everything before this kernel complete, so at most two calls
+    // are ever in flight and the half of the scratch the next quantizer writes is no longer read by anyone).
+    if (p.release_early && warp == 12 && lane == 0) grid_launch_dependents();
     const int quad = warp & 3;
     const int row_in_block = quad * 32 + lane;
     const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -570,6 +606,14 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+  if (p.done != nullptr && tid == 0) {
+    // every thread block of this launch has finished with the quantizer's counters once all have come by here
+    if (atomicAdd(p.done, 1u) == gridDim.x - 1) {
+      unsigned* ready = const_cast<unsigned*>(p.ready);
+      for (int m = 0; m < MAX_MAPS; ++m) atomicExch(ready + m, 0u);
+      atomicExch(p.done, 0u);
+    }
+  }
 }
 
 // ---- host side ----
@@ -632,7 +676,8 @@ int gemm_stream_max_tokens() { return 128 * kMaxPasses; }
 
 // Several weight tensors (each reading one of up to four quantized inputs) in one launch, T <= 128.
 static int launch_gemm_stream_pass(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
-                             int32_t* part, int* flags, cudaStream_t s, int early_release_reserve) {
+                             int32_t* part, int* flags, cudaStream_t s, int early_release_reserve,
+                             const StreamReady* ready, bool last_pass) {
   if (T <= 0 || n_jobs <= 0) return HBL_OK;
   if (T > 128) return HBL_ERR_TOO_LARGE;
   if (n_jobs > MAX_JOBS || n_inputs > MAX_MAPS || n_inputs <= 0) return HBL_ERR_SHAPE;
@@ -690,6 +735,9 @@ static int launch_gemm_stream_pass(const StreamInput* inputs, int n_inputs, cons
   if (p.status == nullptr) return HBL_ERR_CUDA;
   p.T = T;
   p.release_early = early_release_reserve >= 0 ? 1 : 0;
+  p.ready = ready ? ready->ready : nullptr;
+  for (int m = 0; m < MAX_MAPS; ++m) p.ready_target[m] = ready ? ready->target[m] : 0u;
+  p.done = (ready && last_pass) ? ready->done : nullptr;
   // Every CTA that shares a row block writes (and the owner reads) 128 x t_pad partial sums.  Use
   // all SMs only when each one streams several times that in weights; otherwise fewer, fatter
   // CTAs (never fewer than one per row block, which shares nothing).
@@ -736,7 +784,8 @@ static int launch_gemm_stream_pass(const StreamInput* inputs, int n_inputs, cons
 // Up to 512 tokens: the weights stream once per 128 tokens (still far cheaper than expanding them to
 // int8 in HBM for the large-batch kernel, whose tiles would also be mostly padding at these sizes).
 int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
-                             int32_t* part, int* flags, cudaStream_t s, int early_release_reserve) {
+                             int32_t* part, int* flags, cudaStream_t s, int early_release_reserve,
+                             const StreamReady* ready) {
   if (T <= 0 || n_jobs <= 0) return HBL_OK;
   if (T > gemm_stream_max_tokens()) return HBL_ERR_TOO_LARGE;
   if (n_jobs > MAX_JOBS || n_inputs > MAX_MAPS || n_inputs <= 0) return HBL_ERR_SHAPE;
@@ -752,7 +801,8 @@ int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const Stre
       if (jb[j].y) jb[j].y += (size_t)t0 * jobs[j].N;
       if (jb[j].acc_out) jb[j].acc_out += (size_t)t0 * jobs[j].N;
     }
-    const int rc = launch_gemm_stream_pass(in, n_inputs, jb, n_jobs, tn, part, flags + pass * MAX_GRID, s, early_release_reserve);
+    const int rc = launch_gemm_stream_pass(in, n_inputs, jb, n_jobs, tn, part, flags + pass * MAX_GRID, s, early_release_reserve,
+                                           ready, (pass + 1) * 128 >= T);
     if (rc != HBL_OK) return rc;
   }
   return HBL_OK;
@@ -760,10 +810,11 @@ int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const Stre
 
 int launch_gemm_stream(const int8_t* codes, const float* scale, const int32_t* codesum, int T, int K,
                        const void* W_packed, int N, const float* alpha, __nv_bfloat16* y,
-                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s, int early_release_reserve) {
+                       int32_t* acc_out, int32_t* acc_ws, int* counters, cudaStream_t s, int early_release_reserve,
+                       const StreamReady* ready) {
   StreamInput in = {codes, scale, codesum, K};
   StreamJob job = {W_packed, alpha, y, acc_out, N, 0};
-  return launch_gemm_stream_multi(&in, 1, &job, 1, T, acc_ws, counters, s, early_release_reserve);
+  return launch_gemm_stream_multi(&in, 1, &job, 1, T, acc_ws, counters, s, early_release_reserve, ready);
 }
 
 }  // namespace hbl

@@ -31,7 +31,7 @@ def test_wait_runs_out_and_the_library_carries_on():
     W = wl.rows("latent", 21, 2, K, 0, N, "f32")
     o = oracle_layer(x, W, 4, True)
     packed, alpha = hbl.hbl_quantize_weights(torch.from_numpy(W).cuda(), EPS)
-    for path, rows in ((hbl.PATH_TENSOR, T), (hbl.PATH_STREAM, 100)):
+    for path, rows in ((hbl.PATH_TENSOR, T), (hbl.PATH_STREAM, 100), (hbl.PATH_STREAM_OVERLAP, 100)):
         y = hbl.hbl_forward(to_dev(x[:rows], "bf16"), packed, alpha, N, 4, True, EPS, path=path)
         assert hbl.hbl_check_status() == 0
         check_y(y, o["y64"][:rows])
