@@ -104,3 +104,22 @@ def test_layer_back_to_back_calls_equal_plain_streaming_calls(cfg, T):
     assert hbl.hbl_check_status() == 0
     for i in range(3):
         assert torch.equal(ys[i], ref[i]), f"input {i} differs"
+
+
+@pytest.mark.parametrize("dtype,K,had", [(torch.float32, 4096, True), (torch.bfloat16, 1024, True), (torch.float32, 1536, False)])
+def test_layer_back_to_back_without_the_counting_quantizer(dtype, K, had):
+    """Inputs the one-launch quantizer does not serve (fp32, or a transform size outside 2^11..2^14): the mode then
+    rests on the quantizer's completion alone.  Same bar: bit-equality with plain streaming calls."""
+    N, T = 1024, 24
+    g = torch.Generator(device="cuda").manual_seed(K + T)
+    packed, alpha = hbl.hbl_quantize_weights(torch.randn((N, K), device="cuda", generator=g) * 0.02, EPS)
+    xs = [torch.randn((T, K), device="cuda", generator=g).to(dtype) for _ in range(3)]
+    work = hbl.new_workspace(hbl.hbl_workspace_bytes(T, K, N))
+    ref = [hbl.hbl_forward(x, packed, alpha, N, 4, had, EPS, workspace=work, path=hbl.PATH_STREAM).clone() for x in xs]
+    ys = [torch.empty_like(r) for r in ref]
+    for rep in range(60):
+        for i in range(3):
+            hbl.hbl_forward(xs[i], packed, alpha, N, 4, had, EPS, y=ys[i], workspace=work, path=hbl.PATH_STREAM_OVERLAP)
+    assert hbl.hbl_check_status() == 0
+    for i in range(3):
+        assert torch.equal(ys[i], ref[i]), f"input {i} differs"
