@@ -72,8 +72,12 @@ typedef enum {
                               workspace sizes include both); with bf16 inputs the contraction starts on an input's
                               codes as soon as all thread blocks of the quantizer have counted themselves in for it
                               (counters in device memory of the library, 256 workspaces remembered per process).  Any other library call that follows on the stream is
-                              launched as an ordinary kernel and waits for everything before it.  The paper has no
-                              counterpart: this is a launch configuration for back-to-back latency. */
+                              launched as an ordinary kernel and waits for everything before it; a kernel of the
+                              caller's own that is launched with the programmatic-serialization attribute directly
+                              after such a call may start before the call has completed, as after any kernel that
+                              releases its dependents, and has to wait (griddepcontrol.wait) before it reads the
+                              call's outputs.  The paper has no counterpart: this is a launch configuration for
+                              back-to-back latency. */
 } hbl_path_t;
 
 const char* hbl_status_string(int status);
