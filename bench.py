@@ -765,9 +765,14 @@ def main():
         only = [f.split(":") for f in args.only.split(",") if f]
         want = lambda name, T_: (not only) or any(o[0] in name and (len(o) < 2 or int(o[1]) == T_) for o in only)
 
+        # layer and block points are listed in the order they are printed in, but the ones of up to 512 tokens
+        # (latency- and HBM-bound) are measured before the long tensor-bound ones, which leave the clocks under the
+        # power cap for a while
+        plan = []
+
         def L(name, kind, seed, K_, N_, bits, had, T_):
             if want(name, T_):
-                points.append(layer_point(name, kind, seed, K_, N_, bits, had, T_, torch=torch, hbl=hbl, peaks=peaks))
+                plan.append((T_, lambda: layer_point(name, kind, seed, K_, N_, bits, had, T_, torch=torch, hbl=hbl, peaks=peaks)))
 
         # the activation-side kernels first: they are bound by instruction issue, and right after the
         # millisecond-long contractions below the power cap still holds the clocks down
@@ -798,7 +803,13 @@ def main():
                 L(f"config4_a8_N{N_}", "gauss", 4, 4096, N_, 8, False, T_)
         for T_ in ((1, 4, 16, 64, 256, 1024, 4096, 16384, 65536) if full else (1, 16, 256, 4096, 16384)):
             if want("config5_block_7B", T_):
-                points.append(block_point(T_, torch, hbl, peaks))
+                plan.append((T_, lambda T_=T_: block_point(T_, torch, hbl, peaks)))
+        results = [None] * len(plan)
+        for small_first in (True, False):
+            for i, (T_, run) in enumerate(plan):
+                if (T_ <= 512) == small_first:
+                    results[i] = run()
+        points.extend(results)
 
     # the library int8 GEMM runs last: seconds of back-to-back tensor work leave the clocks under the power cap,
     # which the issue-bound points of the sweep would otherwise inherit
