@@ -54,7 +54,12 @@ typedef enum { HBL_F32 = 0, HBL_BF16 = 1 } hbl_dtype_t;
 
 /* Which contraction kernel hbl_forward / hbl_gemm_i32 use. */
 typedef enum {
-  HBL_PATH_AUTO = 0,       /* by token count */
+  HBL_PATH_AUTO = 0,       /* by token count.  Where that gives the streaming kernel, hbl_forward and hbl_block_forward
+                              run the call in the back-to-back mode described under HBL_PATH_STREAM_OVERLAP whenever the
+                              library can see for itself that the statement that mode needs holds: its last launch on the
+                              stream either does not release early, or writes none of the bytes this call reads as
+                              inputs (its outputs and its workspace are compared with this call's inputs as address
+                              ranges).  Otherwise the call is launched as ordinary kernels, as HBL_PATH_STREAM always is. */
   HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers into tensor memory); tokens <= 512 */
   HBL_PATH_TENSOR = 2,     /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
   HBL_PATH_TENSOR_PACKED = 3, /* the same with the INT4 codes kept two per byte between the activation kernel and the
@@ -65,7 +70,7 @@ typedef enum {
                               them (hbl_forward and hbl_block_forward): the contraction releases its programmatic
                               dependents as soon as it has seen its quantizer complete, so the next such call's
                               quantizer runs beside it and the next contraction takes over the SMs as this one's
-                              thread blocks leave.  By this value the caller states that NONE OF THE CALL'S INPUTS
+                              thread blocks leave.  By this value the caller states (HBL_PATH_AUTO checks) that NONE OF THE CALL'S INPUTS
                               IS WRITTEN BY THE LIBRARY CALL ISSUED JUST BEFORE IT ON THE SAME STREAM (they may be
                               read while that call still runs); outputs and workspace are ordered as always.  Calls
                               on one workspace alternate between two halves of the quantizer's scratch (the

@@ -41,7 +41,12 @@ int sm_count() {
 namespace {
 std::mutex g_overlap_mutex;
 constexpr int kStreamSlots = 64, kWorkspaceSlots = 256;
-struct StreamSlot { cudaStream_t s; bool used, early; } g_streams[kStreamSlots] = {};
+constexpr int kMaxRecordedOutputs = 8;
+struct ByteRange { const char* lo; const char* hi; };
+struct StreamSlot {
+  cudaStream_t s; bool used, early;
+  int n_out; ByteRange out[kMaxRecordedOutputs];             // what the early-releasing call writes (its outputs)
+} g_streams[kStreamSlots] = {};
 bool g_stream_overflow = false;       // an early release on a stream that found no slot: every unknown stream counts as early
 struct WorkspaceSlot { const void* ws; bool used; int last; } g_workspaces[kWorkspaceSlots] = {};
 }
@@ -63,9 +68,38 @@ void set_stream_released_early(cudaStream_t s, bool v) {
     if (!g_streams[i].used && free_slot < 0) free_slot = i;
   }
   if (!v && !g_stream_overflow) return;                       // nothing to remember
-  if (free_slot >= 0) g_streams[free_slot] = {s, true, v};
+  if (free_slot >= 0) { g_streams[free_slot] = {}; g_streams[free_slot].s = s; g_streams[free_slot].used = true; g_streams[free_slot].early = v; }
   else if (v) g_stream_overflow = true;
 }
+namespace {
+// The outputs of the early-releasing call just launched on s (called right after set_stream_released_early(s, true)).
+void record_stream_outputs(cudaStream_t s, const ByteRange* out, int n) {
+  std::lock_guard<std::mutex> lock(g_overlap_mutex);
+  for (int i = 0; i < kStreamSlots; ++i)
+    if (g_streams[i].used && g_streams[i].s == s) {
+      g_streams[i].n_out = n < kMaxRecordedOutputs ? n : kMaxRecordedOutputs;
+      for (int k = 0; k < g_streams[i].n_out; ++k) g_streams[i].out[k] = out[k];
+      if (n > kMaxRecordedOutputs) g_streams[i].n_out = -1;   // unknown extent: everything may be written
+      return;
+    }
+}
+// May a quantizer that reads `in` run beside the library's last launch on s?  Yes if that launch does not release
+// its dependents early (the quantizer then starts after it anyway), or if it writes none of these bytes.
+bool inputs_clear_of_last_outputs(cudaStream_t s, const ByteRange* in, int n) {
+  std::lock_guard<std::mutex> lock(g_overlap_mutex);
+  for (int i = 0; i < kStreamSlots; ++i)
+    if (g_streams[i].used && g_streams[i].s == s) {
+      if (!g_streams[i].early) return true;
+      if (g_streams[i].n_out < 0) return false;
+      for (int k = 0; k < g_streams[i].n_out; ++k)
+        for (int j = 0; j < n; ++j)
+          if (in[j].lo < g_streams[i].out[k].hi && g_streams[i].out[k].lo < in[j].hi) return false;
+      return true;
+    }
+  return !g_stream_overflow;
+}
+ByteRange byte_range(const void* p, size_t bytes) { return {static_cast<const char*>(p), static_cast<const char*>(p) + bytes}; }
+}  // namespace
 namespace {
 // Which half of the double-buffered activation scratch the next overlapping call on this workspace writes:
 // the one the call before it did not (0, 1, 0, ...); -1 when the table is full (the call then runs unoverlapped).
@@ -353,8 +387,19 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // back-to-back mode: this call's quantizer may run beside the previous call's contraction, so it writes the half
   // of the scratch that call does not read (no slot left to remember the workspace: an ordinary streaming call)
+  // The automatic path takes the same mode by itself when it can see that the caller's statement holds: the
+  // library's last launch on this stream either does not release early, or writes none of this call's inputs.
+  const size_t x_elem = x_dtype == HBL_BF16 ? 2 : 4;
+  ByteRange ins[3];
+  int n_ins = 0;
+  ins[n_ins++] = byte_range(x, (size_t)tokens * in_dim * x_elem);
+  if (up) ins[n_ins++] = byte_range(up, (size_t)tokens * in_dim * 2);
+  if (gain) ins[n_ins++] = byte_range(gain, (size_t)in_dim * 4);
+  const bool want_overlap = p == HBL_PATH_STREAM_OVERLAP ||
+                            (path == HBL_PATH_AUTO && p == HBL_PATH_STREAM && inputs_clear_of_last_outputs(s, ins, n_ins));
+  const ByteRange outs_written[2] = {byte_range(y, (size_t)tokens * out_dim * 2), byte_range(workspace, w.total)};
   int slot = -1;
-  const int half = (p == HBL_PATH_STREAM_OVERLAP) ? next_overlap_half(workspace, &slot) : -1;
+  const int half = want_overlap ? next_overlap_half(workspace, &slot) : -1;
   const bool overlap = half >= 0;
   OverlapScope scope(overlap);
   char* ws = static_cast<char*>(workspace) + (half == 1 ? w.second_half : 0);
@@ -386,10 +431,12 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
       StreamReady ready = {counters, {0, 0, 0, 0}, counters + 4};
       rc = launch_act_multi_bf16(&job, 1, tokens, bits, eps, zf, zw, s, counters, ready.target);
       if (rc != HBL_OK) return rc;
-      return launch_gemm_stream(codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha,
-                                static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
-                                reinterpret_cast<int*>(ws + w.counters), s,
-                                overlap_reserve((long)tokens * (in_dim / 64 < 32 ? 32 : in_dim / 64)), &ready);
+      rc = launch_gemm_stream(codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha,
+                              static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
+                              reinterpret_cast<int*>(ws + w.counters), s,
+                              overlap_reserve((long)tokens * (in_dim / 64 < 32 ? 32 : in_dim / 64)), &ready);
+      if (rc == HBL_OK) record_stream_outputs(s, outs_written, 2);
+      return rc;
     }
   }
   rc = gain ? launch_norm_act_quant_bf16(x, gain, gain_dtype, norm_eps, tokens, in_dim, bits, eps, codes, scale, cs, nullptr, zf, zw, s, packed)
@@ -399,11 +446,14 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
     if (sp != nullptr) cudaStreamWaitEvent(s, sp->unpacked[0], 0);   // join before reporting the error
     return rc;
   }
-  if (stream_path)
-    return launch_gemm_stream(codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha,
-                              static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
-                              reinterpret_cast<int*>(ws + w.counters), s,
-                              overlap ? overlap_reserve((long)tokens * (in_dim / 64 < 32 ? 32 : in_dim / 64)) : -1);
+  if (stream_path) {
+    rc = launch_gemm_stream(codes, scale, codesum, tokens, in_dim, W_packed, out_dim, alpha,
+                            static_cast<__nv_bfloat16*>(y), nullptr, reinterpret_cast<int32_t*>(ws + w.acc),
+                            reinterpret_cast<int*>(ws + w.counters), s,
+                            overlap ? overlap_reserve((long)tokens * (in_dim / 64 < 32 ? 32 : in_dim / 64)) : -1);
+    if (overlap && rc == HBL_OK) record_stream_outputs(s, outs_written, 2);
+    return rc;
+  }
   HBL_CUDA_OK(cudaStreamWaitEvent(s, sp->unpacked[0], 0));
   return launch_gemm_tensor(codes, packed, scale, tokens, in_dim, w_i8, out_dim, alpha, static_cast<__nv_bfloat16*>(y), nullptr, s);
 }
@@ -550,8 +600,13 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // back-to-back mode (not for the chained feed-forward block, whose second quantizer reads the first launch's
   // outputs): see forward_impl
+  const size_t x_elem = b->x_dtype == HBL_BF16 ? 2 : 4;
+  ByteRange ins[4];
+  for (int i = 0; i < 4; ++i) ins[i] = byte_range(xs[i], xs[i] ? (size_t)T * (i == 3 ? F : H) * x_elem : 0);
+  const bool want_overlap = !chain_ffn && (p == HBL_PATH_STREAM_OVERLAP ||
+                                           (path == HBL_PATH_AUTO && p == HBL_PATH_STREAM && inputs_clear_of_last_outputs(s, ins, 4)));
   int slot = -1;
-  const int half = (p == HBL_PATH_STREAM_OVERLAP && !chain_ffn) ? next_overlap_half(workspace, &slot) : -1;
+  const int half = want_overlap ? next_overlap_half(workspace, &slot) : -1;
   const bool overlap = half >= 0;
   OverlapScope scope(overlap);
   char* ws = static_cast<char*>(workspace) + (half == 1 ? w.second_half : 0);
@@ -614,8 +669,15 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
     if (!chain_ffn) {
       long act_threads = 0;                                   // of the next call's quantizer, which has this call's shape
       for (int i = 0; i < 4; ++i) act_threads += (long)T * (in_dims[i] / 64);
-      return launch_gemm_stream_multi(inputs, 4, jobs, 7, T, part, flags, s, overlap ? overlap_reserve(act_threads) : -1,
-                                      ready.ready != nullptr ? &ready : nullptr);
+      rc = launch_gemm_stream_multi(inputs, 4, jobs, 7, T, part, flags, s, overlap ? overlap_reserve(act_threads) : -1,
+                                    ready.ready != nullptr ? &ready : nullptr);
+      if (overlap && rc == HBL_OK) {
+        ByteRange written[8];
+        for (int i = 0; i < 7; ++i) written[i] = byte_range(ys[i], (size_t)T * out_dims[i] * 2);
+        written[7] = byte_range(workspace, w.total);
+        record_stream_outputs(s, written, 8);
+      }
+      return rc;
     }
     // chained: six projections, then the gating product + quantizer (which also clears the flags again: it
     // starts only when the first launch has completed), then the down projection

@@ -123,3 +123,29 @@ def test_layer_back_to_back_without_the_counting_quantizer(dtype, K, had):
     assert hbl.hbl_check_status() == 0
     for i in range(3):
         assert torch.equal(ys[i], ref[i]), f"input {i} differs"
+
+
+def test_automatic_path_sees_chained_layers():
+    """The automatic path takes the back-to-back mode by itself when the call's inputs are clear of what the call
+    before it writes.  Here they are not: the second layer reads the first layer's output, directly, with nothing in
+    between.  Runs of such pairs, inputs taking turns, must give what two synchronised large-batch calls give."""
+    T, K, N1, N2 = 16, 4096, 4096, 2048
+    g = torch.Generator(device="cuda").manual_seed(321)
+    p1, a1 = hbl.hbl_quantize_weights(torch.randn((N1, K), device="cuda", generator=g) * 0.02, EPS)
+    p2, a2 = hbl.hbl_quantize_weights(torch.randn((N2, N1), device="cuda", generator=g) * 0.02, EPS)
+    xs = [torch.randn((T, K), device="cuda", generator=g).bfloat16() for _ in range(3)]
+    ref = []
+    for x in xs:
+        y1 = hbl.hbl_forward(x, p1, a1, N1, 4, True, EPS, path=hbl.PATH_TENSOR)
+        ref.append(hbl.hbl_forward(y1, p2, a2, N2, 4, True, EPS, path=hbl.PATH_TENSOR).clone())
+    w1 = hbl.new_workspace(hbl.hbl_workspace_bytes(T, K, N1))
+    w2 = hbl.new_workspace(hbl.hbl_workspace_bytes(T, N1, N2))
+    y1 = torch.empty((T, N1), dtype=torch.bfloat16, device="cuda")
+    y2 = [torch.empty((T, N2), dtype=torch.bfloat16, device="cuda") for _ in xs]
+    for rep in range(60):
+        for i, x in enumerate(xs):
+            hbl.hbl_forward(x, p1, a1, N1, 4, True, EPS, y=y1, workspace=w1)          # automatic path
+            hbl.hbl_forward(y1, p2, a2, N2, 4, True, EPS, y=y2[i], workspace=w2)      # reads what the call before wrote
+    assert hbl.hbl_check_status() == 0
+    for i in range(3):
+        assert torch.equal(y2[i], ref[i]), f"input {i} differs"
