@@ -663,7 +663,7 @@ __device__ __forceinline__ void count_block_in(unsigned* counter) {
 }
 
 template <int BITS>
-__global__ void __launch_bounds__(kMultiThreads)
+__global__ void __launch_bounds__(kMultiThreads, 3)
 act_multi_bf16_kernel(const __grid_constant__ ActMultiParams p) {
   extern __shared__ __align__(128) float smem[];
   __shared__ float red_f[16];
