@@ -58,8 +58,9 @@ typedef enum {
                               run the call in the back-to-back mode described under HBL_PATH_STREAM_OVERLAP whenever the
                               library can see for itself that the statement that mode needs holds: its last launch on the
                               stream either does not release early, or writes none of the bytes this call reads as
-                              inputs (its outputs and its workspace are compared with this call's inputs as address
-                              ranges).  Otherwise the call is launched as ordinary kernels, as HBL_PATH_STREAM always is. */
+                              inputs, and does not use this call's workspace unless it is the very same one, base
+                              and size (address ranges of its outputs and its workspace are compared with this call's
+                              inputs and workspace).  Otherwise the call is launched as ordinary kernels, as HBL_PATH_STREAM always is. */
   HBL_PATH_STREAM = 1,     /* weight-streaming kernel (packed weights expanded in registers into tensor memory); tokens <= 512 */
   HBL_PATH_TENSOR = 2,     /* tcgen05 kind::i8 kernel, int32 accumulators in tensor memory */
   HBL_PATH_TENSOR_PACKED = 3, /* the same with the INT4 codes kept two per byte between the activation kernel and the

@@ -83,17 +83,22 @@ void record_stream_outputs(cudaStream_t s, const ByteRange* out, int n) {
       return;
     }
 }
-// May a quantizer that reads `in` run beside the library's last launch on s?  Yes if that launch does not release
-// its dependents early (the quantizer then starts after it anyway), or if it writes none of these bytes.
-bool inputs_clear_of_last_outputs(cudaStream_t s, const ByteRange* in, int n) {
+// May a quantizer that reads `in` and writes into the workspace `ws` run beside the library's last launch on s?
+// Yes if that launch does not release its dependents early (the quantizer then starts after it anyway), or if it
+// writes none of the bytes read and touches none of the workspace -- except that the very same workspace (same
+// base, same size: same layout) is fine, its two halves taking turns.
+bool clear_of_last_call(cudaStream_t s, const ByteRange* in, int n, const ByteRange& ws) {
   std::lock_guard<std::mutex> lock(g_overlap_mutex);
   for (int i = 0; i < kStreamSlots; ++i)
     if (g_streams[i].used && g_streams[i].s == s) {
       if (!g_streams[i].early) return true;
       if (g_streams[i].n_out < 0) return false;
-      for (int k = 0; k < g_streams[i].n_out; ++k)
+      for (int k = 0; k < g_streams[i].n_out; ++k) {
+        const ByteRange& o = g_streams[i].out[k];
         for (int j = 0; j < n; ++j)
-          if (in[j].lo < g_streams[i].out[k].hi && g_streams[i].out[k].lo < in[j].hi) return false;
+          if (in[j].lo < o.hi && o.lo < in[j].hi) return false;
+        if (ws.lo < o.hi && o.lo < ws.hi && !(ws.lo == o.lo && ws.hi == o.hi)) return false;
+      }
       return true;
     }
   return !g_stream_overflow;
@@ -395,9 +400,11 @@ int forward_impl(const void* x, int x_dtype, const void* gain, int gain_dtype, f
   ins[n_ins++] = byte_range(x, (size_t)tokens * in_dim * x_elem);
   if (up) ins[n_ins++] = byte_range(up, (size_t)tokens * in_dim * 2);
   if (gain) ins[n_ins++] = byte_range(gain, (size_t)in_dim * 4);
-  const bool want_overlap = p == HBL_PATH_STREAM_OVERLAP ||
-                            (path == HBL_PATH_AUTO && p == HBL_PATH_STREAM && inputs_clear_of_last_outputs(s, ins, n_ins));
   const ByteRange outs_written[2] = {byte_range(y, (size_t)tokens * out_dim * 2), byte_range(workspace, w.total)};
+  // (the explicit mode is the caller's statement about the inputs; that the workspace is not in use by the call
+  //  before is checked either way)
+  const bool want_overlap = (p == HBL_PATH_STREAM_OVERLAP && clear_of_last_call(s, ins, 0, outs_written[1])) ||
+                            (path == HBL_PATH_AUTO && p == HBL_PATH_STREAM && clear_of_last_call(s, ins, n_ins, outs_written[1]));
   int slot = -1;
   const int half = want_overlap ? next_overlap_half(workspace, &slot) : -1;
   const bool overlap = half >= 0;
@@ -603,8 +610,9 @@ int hbl_block_forward(const hbl_block_t* b, void* workspace, size_t workspace_by
   const size_t x_elem = b->x_dtype == HBL_BF16 ? 2 : 4;
   ByteRange ins[4];
   for (int i = 0; i < 4; ++i) ins[i] = byte_range(xs[i], xs[i] ? (size_t)T * (i == 3 ? F : H) * x_elem : 0);
-  const bool want_overlap = !chain_ffn && (p == HBL_PATH_STREAM_OVERLAP ||
-                                           (path == HBL_PATH_AUTO && p == HBL_PATH_STREAM && inputs_clear_of_last_outputs(s, ins, 4)));
+  const ByteRange ws_range = byte_range(workspace, w.total);
+  const bool want_overlap = !chain_ffn && ((p == HBL_PATH_STREAM_OVERLAP && clear_of_last_call(s, ins, 0, ws_range)) ||
+                                           (path == HBL_PATH_AUTO && p == HBL_PATH_STREAM && clear_of_last_call(s, ins, 4, ws_range)));
   int slot = -1;
   const int half = want_overlap ? next_overlap_half(workspace, &slot) : -1;
   const bool overlap = half >= 0;

@@ -149,3 +149,25 @@ def test_automatic_path_sees_chained_layers():
     assert hbl.hbl_check_status() == 0
     for i in range(3):
         assert torch.equal(y2[i], ref[i]), f"input {i} differs"
+
+
+def test_automatic_path_one_buffer_two_layouts():
+    """One scratch buffer lent to calls of two token counts in turn: same base, different layouts, so the halves of
+    one call are not the halves of the next.  The automatic path has to notice (it compares the whole workspace
+    range with the one the call before used) and must not let the second call's quantizer write while the first
+    call's contraction still reads."""
+    cfg = wl.CONFIG4A
+    N, K = cfg.N, cfg.K
+    g = torch.Generator(device="cuda").manual_seed(99)
+    packed, alpha = hbl.hbl_quantize_weights(torch.randn((N, K), device="cuda", generator=g) * 0.02, EPS)
+    Ts = [16, 64, 5, 64, 16]
+    xs = [torch.randn((T, K), device="cuda", generator=g).bfloat16() for T in Ts]
+    ref = [hbl.hbl_forward(x, packed, alpha, N, cfg.bits, cfg.use_hadamard, EPS, path=hbl.PATH_TENSOR).clone() for x in xs]
+    work = hbl.new_workspace(max(hbl.hbl_workspace_bytes(T, K, N) for T in Ts))
+    ys = [torch.empty_like(r) for r in ref]
+    for rep in range(60):
+        for i, x in enumerate(xs):
+            hbl.hbl_forward(x, packed, alpha, N, cfg.bits, cfg.use_hadamard, EPS, y=ys[i], workspace=work[:hbl.hbl_workspace_bytes(Ts[i], K, N)])
+    assert hbl.hbl_check_status() == 0
+    for i in range(len(xs)):
+        assert torch.equal(ys[i], ref[i]), f"call {i} ({Ts[i]} tokens) differs"
