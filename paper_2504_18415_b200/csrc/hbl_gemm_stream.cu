@@ -78,6 +78,8 @@ struct Params {
   const unsigned* ready;          // nullptr: wait for the kernel before this one as a whole
   unsigned ready_target[MAX_MAPS];
   unsigned* done;                 // non-null: thread blocks of this launch that are through; the last one clears ready[] and done
+  int done_early;                 // count in as soon as the codes producer has read the counters for the last time
+                                  // (single launch per call); else at the end of the kernel (last of several passes)
 };
 struct CodeMaps { CUtensorMap m[MAX_MAPS]; };   // codes [T, K] of each input, box 128 x T_pad, 128-byte swizzle
 
@@ -327,6 +329,16 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
           for (int j = 0; j < KBP; ++j)
             tma_load_2d(c_ring + (size_t)s * C_BYTES + j * (T_PAD * 128), tm_codes, &c_full[s], (kb * KBP + j) * 128, 0);
         }
+      }
+      // This thread is the only one of the CTA that reads the quantizer's counters, and it is through with them.
+      // Once the producers of all CTAs of the launch have come by here, the last one puts the counters back to
+      // zero for the next call that uses this half (here rather than at the end of the kernel: the answer of the
+      // atomic is a trip to L2, which the CTA's last stores should not have to wait for).  Only where the call is
+      // this one launch: with several passes a CTA of an earlier pass may not have read all its counters yet.
+      if (p.done != nullptr && p.done_early && atomicAdd(p.done, 1u) == gridDim.x - 1) {
+        unsigned* ready = const_cast<unsigned*>(p.ready);
+        for (int m = 0; m < MAX_MAPS; ++m) atomicExch(ready + m, 0u);
+        atomicExch(p.done, 0u);
       }
     }
   } else if (warp == 1 || (ISSUERS == 2 && warp == 3)) {
@@ -606,8 +618,9 @@ gemm_stream_kernel(const __grid_constant__ CodeMaps maps, const __grid_constant_
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
-  if (p.done != nullptr && tid == 0) {
-    // every thread block of this launch has finished with the quantizer's counters once all have come by here
+  if (p.done != nullptr && !p.done_early && tid == 0) {
+    // last of several passes: every epilogue of this launch has waited for the passes before it to complete, so
+    // when all CTAs have come by here nobody reads the quantizer's counters any more
     if (atomicAdd(p.done, 1u) == gridDim.x - 1) {
       unsigned* ready = const_cast<unsigned*>(p.ready);
       for (int m = 0; m < MAX_MAPS; ++m) atomicExch(ready + m, 0u);
@@ -677,7 +690,7 @@ int gemm_stream_max_tokens() { return 128 * kMaxPasses; }
 // Several weight tensors (each reading one of up to four quantized inputs) in one launch, T <= 128.
 static int launch_gemm_stream_pass(const StreamInput* inputs, int n_inputs, const StreamJob* jobs, int n_jobs, int T,
                              int32_t* part, int* flags, cudaStream_t s, int early_release_reserve,
-                             const StreamReady* ready, bool last_pass) {
+                             const StreamReady* ready, bool last_pass, bool single_pass) {
   if (T <= 0 || n_jobs <= 0) return HBL_OK;
   if (T > 128) return HBL_ERR_TOO_LARGE;
   if (n_jobs > MAX_JOBS || n_inputs > MAX_MAPS || n_inputs <= 0) return HBL_ERR_SHAPE;
@@ -738,6 +751,7 @@ static int launch_gemm_stream_pass(const StreamInput* inputs, int n_inputs, cons
   p.ready = ready ? ready->ready : nullptr;
   for (int m = 0; m < MAX_MAPS; ++m) p.ready_target[m] = ready ? ready->target[m] : 0u;
   p.done = (ready && last_pass) ? ready->done : nullptr;
+  p.done_early = single_pass ? 1 : 0;
   // Every CTA that shares a row block writes (and the owner reads) 128 x t_pad partial sums.  Use
   // all SMs only when each one streams several times that in weights; otherwise fewer, fatter
   // CTAs (never fewer than one per row block, which shares nothing).
@@ -802,7 +816,7 @@ int launch_gemm_stream_multi(const StreamInput* inputs, int n_inputs, const Stre
       if (jb[j].acc_out) jb[j].acc_out += (size_t)t0 * jobs[j].N;
     }
     const int rc = launch_gemm_stream_pass(in, n_inputs, jb, n_jobs, tn, part, flags + pass * MAX_GRID, s, early_release_reserve,
-                                           ready, (pass + 1) * 128 >= T);
+                                           ready, (pass + 1) * 128 >= T, T <= 128);
     if (rc != HBL_OK) return rc;
   }
   return HBL_OK;
